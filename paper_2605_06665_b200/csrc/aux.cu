@@ -1,0 +1,112 @@
+// Pool-level balance loss (Eqs. 4-5) and the Monte-Carlo constant c (Alg. 1).
+#include "common.cuh"
+
+namespace unipool {
+
+// One block.  counts [L,M] int32, S [L,M] float.
+__global__ void __launch_bounds__(512)
+pool_aux_kernel(const int32_t* __restrict__ counts, const float* __restrict__ S, int L, int M, int T,
+                int k, float alpha, const float* __restrict__ fbar_prev, float* __restrict__ loss,
+                float* __restrict__ coef, float* __restrict__ fbar_out) {
+  __shared__ double red[512];
+  double term = 0.0;
+  for (int i = threadIdx.x; i < M; i += blockDim.x) {
+    double fsum = 0.0, psum = 0.0;
+    for (int l = 0; l < L; ++l) {
+      fsum += (double)counts[(int64_t)l * M + i];
+      psum += (double)S[(int64_t)l * M + i];
+    }
+    const double fbar = fsum / ((double)T * k) / L;       // mean over layers of counts/(T k)
+    const double pbar = psum / (double)T / L;             // mean over layers of S/T
+    const double f_used = fbar_prev ? (double)fbar_prev[i] : fbar;
+    fbar_out[i] = (float)fbar;
+    coef[i] = (float)((double)alpha * M * f_used / ((double)L * T));
+    term += f_used * pbar;
+  }
+  red[threadIdx.x] = term;
+  __syncthreads();
+  for (int o = blockDim.x / 2; o > 0; o >>= 1) {
+    if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) *loss = (float)((double)alpha * M * red[0]);
+}
+
+int aux_launch(unipool_ctx* ctx, const int32_t* counts, const float* S, int L, int M, int T,
+               float alpha, const float* fbar_prev, float* loss, float* coef, float* fbar_out,
+               cudaStream_t s) {
+  pool_aux_kernel<<<1, 512, 0, s>>>(counts, S, L, M, T, ctx->cfg.top_k, alpha, fbar_prev, loss, coef,
+                                    fbar_out);
+  UP_LAUNCH_CHECK();
+  return UNIPOOL_OK;
+}
+
+// ---------------------------------------------------------------- Alg. 1
+// Counter-based generator: a 64-bit mix of (seed, sample, element) gives two
+// uniform 32-bit words, turned into one normal draw by Box-Muller.
+__device__ __forceinline__ uint64_t mix64(uint64_t v) {
+  v += 0x9E3779B97F4A7C15ull;
+  v = (v ^ (v >> 30)) * 0xBF58476D1CE4E5B9ull;
+  v = (v ^ (v >> 27)) * 0x94D049BB133111EBull;
+  return v ^ (v >> 31);
+}
+
+__device__ __forceinline__ float normal_draw(uint64_t seed, uint64_t sample, uint32_t elem) {
+  uint64_t h = mix64(mix64(seed ^ (sample * 0xD1342543DE82EF95ull)) + elem);
+  float u1 = ((uint32_t)(h >> 32) + 1.0f) * (1.0f / 4294967808.0f);   // (0,1)
+  float u2 = (uint32_t)h * (1.0f / 4294967296.0f);
+  return sqrtf(-2.0f * __logf(u1)) * __cosf(6.283185307179586f * u2);
+}
+
+// One thread per sample: keeps the k largest positive components of x, then
+// 1/||top-k(relu(x/||x||))|| = ||x|| / ||top-k(relu(x))||.
+__global__ void __launch_bounds__(256)
+calibrate_kernel(int E, int k, int n_samples, uint64_t seed, double* __restrict__ acc) {
+  const int sidx = blockIdx.x * blockDim.x + threadIdx.x;
+  double inv = 0.0, used = 0.0;
+  if (sidx < n_samples) {
+    float top[UNIPOOL_MAX_TOPK];
+#pragma unroll
+    for (int j = 0; j < UNIPOOL_MAX_TOPK; ++j) top[j] = 0.f;
+    float ss = 0.f;
+    for (int e = 0; e < E; ++e) {
+      float v = normal_draw(seed, (uint64_t)sidx, (uint32_t)e);
+      ss = fmaf(v, v, ss);
+      float r = fmaxf(v, 0.f);
+      // insertion into the descending list top[0..k)
+#pragma unroll
+      for (int j = 0; j < UNIPOOL_MAX_TOPK; ++j) {
+        if (j < k && r > top[j]) { float tmp = top[j]; top[j] = r; r = tmp; }
+      }
+    }
+    float ts = 0.f;
+#pragma unroll
+    for (int j = 0; j < UNIPOOL_MAX_TOPK; ++j) if (j < k) ts = fmaf(top[j], top[j], ts);
+    if (ts > 0.f) { inv = (double)(sqrtf(ss) / sqrtf(ts)); used = 1.0; }
+  }
+  __shared__ double r0[256], r1[256];
+  r0[threadIdx.x] = inv;
+  r1[threadIdx.x] = used;
+  __syncthreads();
+  for (int o = 128; o > 0; o >>= 1) {
+    if (threadIdx.x < o) { r0[threadIdx.x] += r0[threadIdx.x + o]; r1[threadIdx.x] += r1[threadIdx.x + o]; }
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) { atomicAdd(&acc[0], r0[0]); atomicAdd(&acc[1], r1[0]); }
+}
+
+int calibrate_launch(unipool_ctx* ctx, int E, int k, int n_samples, uint64_t seed, float* c_out,
+                     cudaStream_t s) {
+  double* acc = ctx->ws.dsigma_acc;     // two doubles, zero between calls
+  calibrate_kernel<<<(n_samples + 255) / 256, 256, 0, s>>>(E, k, n_samples, seed, acc);
+  UP_LAUNCH_CHECK();
+  double host[2];
+  UP_CUDA(cudaMemcpyAsync(host, acc, sizeof(host), cudaMemcpyDeviceToHost, s));
+  UP_CUDA(cudaMemsetAsync(acc, 0, sizeof(host), s));
+  UP_CUDA(cudaStreamSynchronize(s));
+  UP_REQUIRE(host[1] > 0.0, UNIPOOL_ERR_DEVICE_CHECK, "calibrate_c: no usable sample");
+  *c_out = (float)(host[0] / host[1]);
+  return UNIPOOL_OK;
+}
+
+}  // namespace unipool

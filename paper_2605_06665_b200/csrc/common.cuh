@@ -1,0 +1,144 @@
+// Shared host/device declarations of the UniPool library (internal header).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "unipool.h"
+
+namespace unipool {
+
+// ---------------------------------------------------------------- errors
+void set_error(const char* fmt, ...);
+
+#define UP_REQUIRE(cond, code, ...)      \
+  do {                                   \
+    if (!(cond)) {                       \
+      unipool::set_error(__VA_ARGS__);   \
+      return (code);                     \
+    }                                    \
+  } while (0)
+
+#define UP_CUDA(call)                                                                  \
+  do {                                                                                 \
+    cudaError_t e__ = (call);                                                          \
+    if (e__ != cudaSuccess) {                                                          \
+      unipool::set_error("%s failed: %s (%s:%d)", #call, cudaGetErrorString(e__), __FILE__, \
+                         __LINE__);                                                    \
+      return UNIPOOL_ERR_CUDA;                                                         \
+    }                                                                                  \
+  } while (0)
+
+#define UP_LAUNCH_CHECK()                                                              \
+  do {                                                                                 \
+    cudaError_t e__ = cudaGetLastError();                                              \
+    if (e__ != cudaSuccess) {                                                          \
+      unipool::set_error("kernel launch failed: %s (%s:%d)", cudaGetErrorString(e__),  \
+                         __FILE__, __LINE__);                                          \
+      return UNIPOOL_ERR_CUDA;                                                         \
+    }                                                                                  \
+  } while (0)
+
+// ---------------------------------------------------------------- workspace
+// Fixed layout of the caller's workspace; every region is 256-byte aligned.
+struct Workspace {
+  int32_t* status;        // [4]   device status word (+ spare)
+  int32_t* route_counts;  // [MAX_EXPERTS] self-cleaning accumulators of route
+  double*  route_sums;    // [MAX_EXPERTS]
+  uint32_t* tickets;      // [8]   "last block done" counters, self-cleaning
+  double*  dsigma_acc;    // [2]   self-cleaning accumulator of route_bwd / calibrate_c
+  int32_t* block_hist;    // [dispatch_blocks, MAX_EXPERTS]
+  float*   dz;            // [max_tokens, pool_size] route_bwd scratch
+  void*    dXp;           // [row_capacity, d] expert_bwd scratch (ctx dtype)
+  size_t   bytes;         // total
+};
+
+constexpr int kDispatchChunkTokens = 64;   // tokens per dispatch block
+
+Workspace carve_workspace(const unipool_config& cfg, void* base);
+
+}  // namespace unipool
+
+struct unipool_ctx {
+  unipool_config cfg;
+  unipool::Workspace ws;
+  int device;
+  int sm_count;
+  int64_t row_capacity;
+  size_t elem_bytes;
+  void* tmap_cache;   // opaque, owned by the tensor-core GEMM module
+};
+
+namespace unipool {
+
+// ---------------------------------------------------------------- element helpers
+__device__ __forceinline__ float to_f32(float v) { return v; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) {
+  return __float2bfloat16_rn(v);
+}
+
+__device__ __forceinline__ float silu_f(float a) { return a / (1.0f + __expf(-a)); }
+__device__ __forceinline__ float silu_grad_f(float a) {
+  float sig = 1.0f / (1.0f + __expf(-a));
+  return sig * (1.0f + a * (1.0f - sig));
+}
+
+// status codes written by kernels into ws.status[0]
+constexpr int kStatusTimeout = 1;
+constexpr int kStatusCheck = 2;
+
+// ---------------------------------------------------------------- module entry points
+int route_launch(unipool_ctx*, const void* x, int T, const float* W_r, float sigma,
+                 const float* bias, int n_experts, int32_t* idx, float* gate, int32_t* counts,
+                 float* score_sum, float* znorm, float* z_saved, cudaStream_t);
+int route_bwd_launch(unipool_ctx*, const void* x, int T, const float* W_r, float sigma,
+                     int n_experts, const float* znorm, const float* z_saved, const int32_t* idx,
+                     const float* dgate, const float* coef, void* dx, float* dW_r, float* dsigma,
+                     cudaStream_t);
+int dispatch_launch(unipool_ctx*, const void* x, int T, const int32_t* idx, int n_experts,
+                    int32_t* offsets, int32_t* row_of, int32_t* token_of, int32_t* tile_expert,
+                    void* Xp, cudaStream_t);
+int combine_launch(unipool_ctx*, const void* Yp, const int32_t* row_of, const float* gate, int T,
+                   const void* residual, void* y, cudaStream_t);
+int combine_bwd_launch(unipool_ctx*, const void* dy, int T, const int32_t* row_of,
+                       const float* gate, const int32_t* token_of, const int32_t* offsets,
+                       int n_experts, const void* Yp, void* dYp, float* dgate, cudaStream_t);
+int unpermute_sum_launch(unipool_ctx*, const void* dXp, const int32_t* row_of, int T,
+                         const void* residual, void* dx, cudaStream_t);
+int aux_launch(unipool_ctx*, const int32_t* counts, const float* S, int L, int n_experts, int T,
+               float alpha, const float* fbar_prev, float* loss, float* coef, float* fbar_out,
+               cudaStream_t);
+int calibrate_launch(unipool_ctx*, int n_experts, int top_k, int n_samples, uint64_t seed,
+                     float* c_out, cudaStream_t);
+
+// grouped GEMMs: CUDA-core path (fp32 mode) and tcgen05 path (bf16 mode)
+struct ExpertFwdArgs {
+  const void* Xp; const int32_t* offsets; const int32_t* tile_expert;
+  const void* W_gu; const void* W_down; int expert_base; int n_experts;
+  void* GU; void* A; void* Yp;
+};
+struct ExpertBwdArgs {
+  const int32_t* offsets; const int32_t* tile_expert;
+  const void* Xp; const void* GU; const void* A; const void* W_gu; const void* W_down;
+  int expert_base; int n_experts;
+  const void* dYp; void* dGU; void* dXp; float* dW_gu; float* dW_down; bool wgrad;
+};
+struct PoolWgradArgs {
+  int n_layers; int64_t layer_stride_rows; const int32_t* offsets;
+  const void* Xp; const void* A; const void* dYp; const void* dGU;
+  int expert_base; int n_experts; float* dW_gu; float* dW_down;
+};
+int expert_fwd_simt(unipool_ctx*, const ExpertFwdArgs&, cudaStream_t);
+int expert_bwd_simt(unipool_ctx*, const ExpertBwdArgs&, cudaStream_t);
+int pool_wgrad_simt(unipool_ctx*, const PoolWgradArgs&, cudaStream_t);
+int expert_fwd_tc(unipool_ctx*, const ExpertFwdArgs&, cudaStream_t);
+int expert_bwd_tc(unipool_ctx*, const ExpertBwdArgs&, cudaStream_t);
+int pool_wgrad_tc(unipool_ctx*, const PoolWgradArgs&, cudaStream_t);
+int tc_module_init(unipool_ctx*);
+void tc_module_destroy(unipool_ctx*);
+
+}  // namespace unipool

@@ -1,0 +1,347 @@
+// Token permute into expert-contiguous order and its inverse (combine), forward
+// and backward.  All data movement is in 16-byte vectors; one warp moves one row.
+#include "common.cuh"
+
+namespace unipool {
+
+// ---------------------------------------------------------------- maps
+// Block b owns tokens [b*CH, (b+1)*CH); one warp per block so that the stable
+// (token-major) order inside the chunk is the lane order.
+__global__ void __launch_bounds__(32)
+dispatch_hist_kernel(const int32_t* __restrict__ idx, int T, int k, int M, int32_t* __restrict__ block_hist,
+                     int32_t* __restrict__ status) {
+  extern __shared__ int hist[];
+  const int lane = threadIdx.x;
+  for (int i = lane; i < M; i += 32) hist[i] = 0;
+  __syncwarp();
+  const int64_t a_begin = (int64_t)blockIdx.x * kDispatchChunkTokens * k;
+  const int64_t a_end = min((int64_t)T * k, a_begin + (int64_t)kDispatchChunkTokens * k);
+  for (int64_t a = a_begin + lane; a < a_end; a += 32) {
+    int e = idx[a];
+    if (e < 0 || e >= M) {          // corrupt routing table: record it, drop the assignment
+      if (atomicCAS(status, 0, kStatusCheck) == 0) { status[1] = 10; status[2] = e; }
+      continue;
+    }
+    atomicAdd(&hist[e], 1);
+  }
+  __syncwarp();
+  for (int i = lane; i < M; i += 32) block_hist[(int64_t)blockIdx.x * M + i] = hist[i];
+}
+
+// One block: per-expert totals -> padded exclusive scan -> per-(block, expert) bases.
+// block_hist[b][e] is replaced by the first row of block b's assignments to e.
+__global__ void __launch_bounds__(512)
+dispatch_scan_kernel(int32_t* __restrict__ block_hist, int n_blocks, int M, int row_capacity,
+                     int32_t* __restrict__ offsets, int32_t* __restrict__ token_of,
+                     int32_t* __restrict__ tile_expert) {
+  __shared__ int padded[UNIPOOL_MAX_EXPERTS];
+  __shared__ int start[UNIPOOL_MAX_EXPERTS + 1];
+  __shared__ int total_s[UNIPOOL_MAX_EXPERTS];
+  const int e = threadIdx.x;
+  int total = 0;
+  if (e < M) {
+    for (int b = 0; b < n_blocks; ++b) total += block_hist[(int64_t)b * M + e];
+    total_s[e] = total;
+    padded[e] = (total + UNIPOOL_ROW_ALIGN - 1) / UNIPOOL_ROW_ALIGN * UNIPOOL_ROW_ALIGN;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int run = 0;
+    for (int i = 0; i < M; ++i) { start[i] = run; run += padded[i]; }
+    start[M] = run;
+  }
+  __syncthreads();
+  if (e < M) offsets[e] = start[e];
+  if (e == 0) offsets[M] = start[M];
+  if (e < M) {
+    int run = start[e];
+    for (int b = 0; b < n_blocks; ++b) {
+      int h = block_hist[(int64_t)b * M + e];
+      block_hist[(int64_t)b * M + e] = run;
+      run += h;
+    }
+  }
+  // pad rows of every group, rows beyond the last group, tile -> expert table
+  const int used = start[M];
+  for (int g = 0; g < M; ++g) {
+    int lo = start[g] + total_s[g], hi = start[g + 1];
+    for (int r = lo + threadIdx.x; r < hi; r += blockDim.x) token_of[r] = -1;
+    for (int tl = start[g] / UNIPOOL_ROW_ALIGN + threadIdx.x; tl < start[g + 1] / UNIPOOL_ROW_ALIGN; tl += blockDim.x)
+      tile_expert[tl] = g;
+  }
+  for (int r = used + threadIdx.x; r < row_capacity; r += blockDim.x) token_of[r] = -1;
+  for (int tl = used / UNIPOOL_ROW_ALIGN + threadIdx.x; tl < row_capacity / UNIPOOL_ROW_ALIGN; tl += blockDim.x)
+    tile_expert[tl] = -1;
+}
+
+__global__ void __launch_bounds__(32)
+dispatch_rank_kernel(const int32_t* __restrict__ idx, int T, int k, int M,
+                     const int32_t* __restrict__ block_base, int32_t* __restrict__ row_of,
+                     int32_t* __restrict__ token_of) {
+  extern __shared__ int next_row[];
+  const int lane = threadIdx.x;
+  for (int i = lane; i < M; i += 32) next_row[i] = block_base[(int64_t)blockIdx.x * M + i];
+  __syncwarp();
+  const int64_t a_begin = (int64_t)blockIdx.x * kDispatchChunkTokens * k;
+  const int64_t a_end = min((int64_t)T * k, a_begin + (int64_t)kDispatchChunkTokens * k);
+  for (int64_t a0 = a_begin; a0 < a_end; a0 += 32) {
+    const int64_t a = a0 + lane;
+    const bool live = a < a_end;
+    int e = live ? idx[a] : -1;
+    const bool ok = live && e >= 0 && e < M;
+    if (!ok) e = -1 - lane;                                  // unique key: matches nobody
+    const unsigned peers = __match_any_sync(0xffffffffu, e);
+    const int rank = __popc(peers & ((1u << lane) - 1u));
+    int row = -1;
+    if (ok) row = next_row[e] + rank;
+    __syncwarp();
+    if (ok && rank == 0) next_row[e] += __popc(peers);       // leader = lowest lane of the peer set
+    __syncwarp();
+    if (live) row_of[a] = row;
+    if (ok) token_of[row] = (int)(a / k);
+  }
+}
+
+// ---------------------------------------------------------------- row movers
+// Vector type: 16 bytes.
+template <typename T>
+__device__ __forceinline__ void zero16(uint4& v) { v = make_uint4(0, 0, 0, 0); }
+
+// Xp[r] = x[token_of[r]]  (zero on pad rows), one warp per row, rows < offsets[M].
+__global__ void __launch_bounds__(256)
+gather_rows_kernel(const uint4* __restrict__ x, const int32_t* __restrict__ token_of,
+                   const int32_t* __restrict__ offsets_end, uint4* __restrict__ Xp, int row_vecs,
+                   int row_capacity) {
+  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+  const int used = *offsets_end;
+  for (int r = blockIdx.x * 8 + warp; r < used; r += gridDim.x * 8) {
+    const int t = token_of[r];
+    uint4* dst = Xp + (int64_t)r * row_vecs;
+    if (t >= 0) {
+      const uint4* src = x + (int64_t)t * row_vecs;
+      for (int v = lane; v < row_vecs; v += 32) dst[v] = __ldg(src + v);
+    } else {
+      for (int v = lane; v < row_vecs; v += 32) dst[v] = make_uint4(0, 0, 0, 0);
+    }
+  }
+}
+
+template <typename T> struct Vec16;
+template <> struct Vec16<float> {
+  static constexpr int N = 4;
+  __device__ static void unpack(const uint4& v, float* f) {
+    f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y);
+    f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
+  }
+  __device__ static uint4 pack(const float* f) {
+    return make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]), __float_as_uint(f[2]), __float_as_uint(f[3]));
+  }
+};
+template <> struct Vec16<__nv_bfloat16> {
+  static constexpr int N = 8;
+  __device__ static void unpack(const uint4& v, float* f) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      f[2 * i] = __uint_as_float(w[i] << 16);
+      f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+  }
+  __device__ static uint4 pack(const float* f) {
+    uint32_t w[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      __nv_bfloat162 p = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+      w[i] = *reinterpret_cast<uint32_t*>(&p);
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+  }
+};
+
+// y[t] = (residual[t]) + sum_j gate[t,j] * Yp[row_of[t,j]]   (gate == NULL: unit weights)
+template <typename T>
+__global__ void __launch_bounds__(256)
+combine_kernel(const uint4* __restrict__ Yp, const int32_t* __restrict__ row_of,
+               const float* __restrict__ gate, const uint4* __restrict__ residual,
+               uint4* __restrict__ y, int n_tokens, int k, int row_vecs) {
+  constexpr int N = Vec16<T>::N;
+  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+  for (int t = blockIdx.x * 8 + warp; t < n_tokens; t += gridDim.x * 8) {
+    int rows[UNIPOOL_MAX_TOPK];
+    float g[UNIPOOL_MAX_TOPK];
+    for (int j = 0; j < k; ++j) {
+      rows[j] = row_of[(int64_t)t * k + j];
+      g[j] = gate ? gate[(int64_t)t * k + j] : 1.f;
+    }
+    for (int v = lane; v < row_vecs; v += 32) {
+      float acc[N];
+      if (residual) {
+        Vec16<T>::unpack(__ldg(residual + (int64_t)t * row_vecs + v), acc);
+      } else {
+#pragma unroll
+        for (int i = 0; i < N; ++i) acc[i] = 0.f;
+      }
+      for (int j = 0; j < k; ++j) {
+        if (rows[j] < 0) continue;
+        float f[N];
+        Vec16<T>::unpack(__ldg(Yp + (int64_t)rows[j] * row_vecs + v), f);
+#pragma unroll
+        for (int i = 0; i < N; ++i) acc[i] = fmaf(g[j], f[i], acc[i]);
+      }
+      y[(int64_t)t * row_vecs + v] = Vec16<T>::pack(acc);
+    }
+  }
+}
+
+// dYp[r] = gate(r) * dy[token_of[r]] (zero on pad rows) for rows < offsets[M];
+// the gate of a row is found through row_of: slot j of token t with row_of[t,j] == r.
+template <typename T>
+__global__ void __launch_bounds__(256)
+scale_gather_kernel(const uint4* __restrict__ dy, const int32_t* __restrict__ token_of,
+                    const int32_t* __restrict__ row_of, const float* __restrict__ gate,
+                    const int32_t* __restrict__ offsets_end, uint4* __restrict__ dYp, int k,
+                    int row_vecs) {
+  constexpr int N = Vec16<T>::N;
+  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+  const int used = *offsets_end;
+  for (int r = blockIdx.x * 8 + warp; r < used; r += gridDim.x * 8) {
+    const int t = token_of[r];
+    uint4* dst = dYp + (int64_t)r * row_vecs;
+    if (t < 0) {
+      for (int v = lane; v < row_vecs; v += 32) dst[v] = make_uint4(0, 0, 0, 0);
+      continue;
+    }
+    float g = 0.f;
+    for (int j = 0; j < k; ++j)
+      if (row_of[(int64_t)t * k + j] == r) g = gate[(int64_t)t * k + j];
+    const uint4* src = dy + (int64_t)t * row_vecs;
+    for (int v = lane; v < row_vecs; v += 32) {
+      float f[N];
+      Vec16<T>::unpack(__ldg(src + v), f);
+#pragma unroll
+      for (int i = 0; i < N; ++i) f[i] *= g;
+      dst[v] = Vec16<T>::pack(f);
+    }
+  }
+}
+
+// dgate[t,j] = <dy[t], Yp[row_of[t,j]]>, one warp per token.
+template <typename T>
+__global__ void __launch_bounds__(256)
+dgate_kernel(const uint4* __restrict__ dy, const uint4* __restrict__ Yp,
+             const int32_t* __restrict__ row_of, float* __restrict__ dgate, int n_tokens, int k,
+             int row_vecs) {
+  constexpr int N = Vec16<T>::N;
+  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+  for (int t = blockIdx.x * 8 + warp; t < n_tokens; t += gridDim.x * 8) {
+    float acc[UNIPOOL_MAX_TOPK];
+    int rows[UNIPOOL_MAX_TOPK];
+#pragma unroll
+    for (int j = 0; j < UNIPOOL_MAX_TOPK; ++j) { acc[j] = 0.f; rows[j] = j < k ? row_of[(int64_t)t * k + j] : -1; }
+    for (int v = lane; v < row_vecs; v += 32) {
+      float a[N];
+      Vec16<T>::unpack(__ldg(dy + (int64_t)t * row_vecs + v), a);
+#pragma unroll
+      for (int j = 0; j < UNIPOOL_MAX_TOPK; ++j) {
+        if (rows[j] < 0) continue;
+        float f[N];
+        Vec16<T>::unpack(__ldg(Yp + (int64_t)rows[j] * row_vecs + v), f);
+#pragma unroll
+        for (int i = 0; i < N; ++i) acc[j] = fmaf(a[i], f[i], acc[j]);
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < UNIPOOL_MAX_TOPK; ++j) {
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], o);
+      if (lane == 0 && j < k) dgate[(int64_t)t * k + j] = acc[j];
+    }
+  }
+}
+
+__global__ void dispatch_empty_kernel(int32_t* offsets, int32_t* token_of, int32_t* tile_expert, int M,
+                                      int row_capacity) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i <= M) offsets[i] = 0;
+  if (i < row_capacity) token_of[i] = -1;
+  if (i < row_capacity / UNIPOOL_ROW_ALIGN) tile_expert[i] = -1;
+}
+
+static int row_mover_grid(const unipool_ctx* ctx, int64_t rows) {
+  int64_t want = (rows + 7) / 8;
+  int64_t cap = (int64_t)ctx->sm_count * 8;      // 8 resident 256-thread blocks per SM
+  return (int)(want < 1 ? 1 : (want < cap ? want : cap));
+}
+
+int dispatch_launch(unipool_ctx* ctx, const void* x, int T, const int32_t* idx, int M,
+                    int32_t* offsets, int32_t* row_of, int32_t* token_of, int32_t* tile_expert,
+                    void* Xp, cudaStream_t s) {
+  const int k = ctx->cfg.top_k, d = ctx->cfg.d_model;
+  const int cap = (int)ctx->row_capacity;
+  if (T == 0) {
+    dispatch_empty_kernel<<<(cap + 255) / 256, 256, 0, s>>>(offsets, token_of, tile_expert, M, cap);
+    UP_LAUNCH_CHECK();
+    return UNIPOOL_OK;
+  }
+  const int n_blocks = (T + kDispatchChunkTokens - 1) / kDispatchChunkTokens;
+  int32_t* bh = ctx->ws.block_hist;
+  dispatch_hist_kernel<<<n_blocks, 32, M * sizeof(int), s>>>(idx, T, k, M, bh, ctx->ws.status);
+  UP_LAUNCH_CHECK();
+  dispatch_scan_kernel<<<1, 512, 0, s>>>(bh, n_blocks, M, cap, offsets, token_of, tile_expert);
+  UP_LAUNCH_CHECK();
+  dispatch_rank_kernel<<<n_blocks, 32, M * sizeof(int), s>>>(idx, T, k, M, bh, row_of, token_of);
+  UP_LAUNCH_CHECK();
+  const int row_vecs = (int)((size_t)d * ctx->elem_bytes / 16);
+  gather_rows_kernel<<<row_mover_grid(ctx, cap), 256, 0, s>>>(
+      static_cast<const uint4*>(x), token_of, offsets + M, static_cast<uint4*>(Xp), row_vecs, cap);
+  UP_LAUNCH_CHECK();
+  return UNIPOOL_OK;
+}
+
+int combine_launch(unipool_ctx* ctx, const void* Yp, const int32_t* row_of, const float* gate, int T,
+                   const void* residual, void* y, cudaStream_t s) {
+  if (T == 0) return UNIPOOL_OK;
+  const int k = ctx->cfg.top_k;
+  const int row_vecs = (int)((size_t)ctx->cfg.d_model * ctx->elem_bytes / 16);
+  const int grid = row_mover_grid(ctx, T);
+  if (ctx->cfg.dtype == UNIPOOL_BF16)
+    combine_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>(static_cast<const uint4*>(Yp), row_of, gate,
+        static_cast<const uint4*>(residual), static_cast<uint4*>(y), T, k, row_vecs);
+  else
+    combine_kernel<float><<<grid, 256, 0, s>>>(static_cast<const uint4*>(Yp), row_of, gate,
+        static_cast<const uint4*>(residual), static_cast<uint4*>(y), T, k, row_vecs);
+  UP_LAUNCH_CHECK();
+  return UNIPOOL_OK;
+}
+
+int combine_bwd_launch(unipool_ctx* ctx, const void* dy, int T, const int32_t* row_of,
+                       const float* gate, const int32_t* token_of, const int32_t* offsets, int M,
+                       const void* Yp, void* dYp, float* dgate, cudaStream_t s) {
+  if (T == 0) return UNIPOOL_OK;
+  const int k = ctx->cfg.top_k;
+  const int row_vecs = (int)((size_t)ctx->cfg.d_model * ctx->elem_bytes / 16);
+  const int g1 = row_mover_grid(ctx, ctx->row_capacity), g2 = row_mover_grid(ctx, T);
+  if (ctx->cfg.dtype == UNIPOOL_BF16) {
+    scale_gather_kernel<__nv_bfloat16><<<g1, 256, 0, s>>>(static_cast<const uint4*>(dy), token_of, row_of,
+        gate, offsets + M, static_cast<uint4*>(dYp), k, row_vecs);
+    UP_LAUNCH_CHECK();
+    dgate_kernel<__nv_bfloat16><<<g2, 256, 0, s>>>(static_cast<const uint4*>(dy), static_cast<const uint4*>(Yp),
+        row_of, dgate, T, k, row_vecs);
+  } else {
+    scale_gather_kernel<float><<<g1, 256, 0, s>>>(static_cast<const uint4*>(dy), token_of, row_of, gate,
+        offsets + M, static_cast<uint4*>(dYp), k, row_vecs);
+    UP_LAUNCH_CHECK();
+    dgate_kernel<float><<<g2, 256, 0, s>>>(static_cast<const uint4*>(dy), static_cast<const uint4*>(Yp),
+        row_of, dgate, T, k, row_vecs);
+  }
+  UP_LAUNCH_CHECK();
+  return UNIPOOL_OK;
+}
+
+int unpermute_sum_launch(unipool_ctx* ctx, const void* dXp, const int32_t* row_of, int T,
+                         const void* residual, void* dx, cudaStream_t s) {
+  // dx_t = residual_t + sum_j dXp[row_of[t,j]]: the combine kernel with unit weights
+  return combine_launch(ctx, dXp, row_of, nullptr, T, residual, dx, s);
+}
+
+}  // namespace unipool

@@ -1,0 +1,168 @@
+"""A residual stack of UniPool MoE layers driven through the C-ABI library.
+
+``UniPoolStack`` owns the device buffers (PyTorch tensors) and issues, per layer,
+the library calls route -> dispatch -> expert_fwd -> combine (forward), then
+pool_aux_loss, then expert_bwd -> route_bwd per layer in reverse (backward).
+It contains no arithmetic of its own: every tensor it returns was written by a
+CUDA kernel of the library.
+
+Layer l computes x_{l+1} = x_l + sum_{i in top-k} g_{l,i}(x_l) e_i(x_l)  (Eq. 2),
+all layers sharing one pool of experts; with ``private = E`` layer l instead
+owns pool experts [E*l, E*(l+1)) (the layer-private layout of Eq. 1) and the
+balance loss is the per-layer loss of Eq. 3 summed over layers.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from . import binding as B
+
+
+class UniPoolStack:
+    def __init__(self, L, d, f, M, k, T, dtype="bf16", private=0, c=1.0, eps=1e-6, alpha=1e-2,
+                 device="cuda", deferred_wgrad=False):
+        self.L, self.d, self.f, self.M, self.k, self.T = L, d, f, M, k, T
+        self.private = private
+        self.m = private if private else M                 # experts one router scores
+        self.alpha = alpha
+        self.c, self.eps = c, eps
+        self.deferred_wgrad = deferred_wgrad and not private
+        self.device = torch.device(device)
+        self.tdtype = torch.bfloat16 if dtype == "bf16" else torch.float32
+        self.cfg = B.make_config(d, f, M, k, L, T, B.BF16 if dtype == "bf16" else B.FP32, eps, c)
+        self.ctx = B.Context(self.cfg, self.device)
+        cap = self.ctx.row_capacity
+        self.cap = cap
+        dev, td = self.device, self.tdtype
+        i32, f32 = torch.int32, torch.float32
+        e = lambda *shape, dtype=td: torch.empty(*shape, dtype=dtype, device=dev)
+        # parameters
+        self.W_gu = e(M, 2 * f, d)
+        self.W_down = e(M, d, f)
+        self.W_r = e(L, self.m, d, dtype=f32)
+        self.sigma = [1.0] * L
+        self.bias = None                                   # [L, m] float or None
+        # gradients (fp32; one buffer per pool expert, shared by all layers)
+        self.dW_gu = torch.zeros(M, 2 * f, d, dtype=f32, device=dev)
+        self.dW_down = torch.zeros(M, d, f, dtype=f32, device=dev)
+        self.dW_r = torch.zeros(L, self.m, d, dtype=f32, device=dev)
+        self.dsigma = torch.zeros(L, dtype=f32, device=dev)
+        # activations and routing state kept for backward
+        self.x = e(L + 1, T, d)
+        self.idx = e(L, T, k, dtype=i32)
+        self.gate = e(L, T, k, dtype=f32)
+        self.counts = e(L, self.m, dtype=i32)
+        self.score_sum = e(L, self.m, dtype=f32)
+        self.znorm = e(L, T, dtype=f32)
+        self.z = e(L, T, self.m, dtype=f32)
+        self.offsets = e(L, self.m + 1, dtype=i32)
+        self.row_of = e(L, T, k, dtype=i32)
+        self.token_of = e(L, cap, dtype=i32)
+        self.tile_expert = e(L, cap // B.ROW_ALIGN, dtype=i32)
+        self.Xp = e(L, cap, d)
+        self.GU = e(L, cap, 2 * f)
+        self.A = e(L, cap, f)
+        self.Yp = e(L, cap, d)
+        nb = L if self.deferred_wgrad else 1
+        self.dYp = e(nb, cap, d)
+        self.dGU = e(nb, cap, 2 * f)
+        self.dx = e(2, T, d)                               # ping-pong dx_{l+1} -> dx_l
+        self.dgate = e(T, k, dtype=f32)
+        # balance loss
+        n_aux = L if private else 1
+        self.loss = torch.zeros(n_aux, dtype=f32, device=dev)
+        self.coef = e(n_aux, self.m, dtype=f32)
+        self.fbar = e(n_aux, self.m, dtype=f32)
+
+    # ------------------------------------------------------------------ parameters
+    def load(self, pool, routers):
+        """pool: dict(W_gate [M,f,d], W_up [M,f,d], W_down [M,d,f]); routers: list of
+        dict(W_r [m,d], sigma, bias|None) - numpy float32 arrays (host)."""
+        f = self.f
+        self.W_gu[:, :f].copy_(torch.from_numpy(pool["W_gate"]))
+        self.W_gu[:, f:].copy_(torch.from_numpy(pool["W_up"]))
+        self.W_down.copy_(torch.from_numpy(pool["W_down"]))
+        for l, r in enumerate(routers):
+            self.W_r[l].copy_(torch.from_numpy(r["W_r"]))
+            self.sigma[l] = float(r["sigma"])
+        if routers[0].get("bias") is not None:
+            self.bias = torch.from_numpy(np.stack([r["bias"] for r in routers])).to(self.device)
+        torch.cuda.synchronize(self.device)
+
+    def base(self, l):
+        return self.private * l if self.private else 0
+
+    def zero_grad(self):
+        self.dW_gu.zero_(); self.dW_down.zero_(); self.dW_r.zero_(); self.dsigma.zero_()
+
+    # ------------------------------------------------------------------ forward
+    def forward_layer(self, l, T=None):
+        T = self.T if T is None else T
+        c = self.ctx
+        bias = None if self.bias is None else self.bias[l]
+        c.route(self.x[l], T, self.W_r[l], self.sigma[l], bias, self.m, self.idx[l], self.gate[l],
+                self.counts[l], self.score_sum[l], self.znorm[l], self.z[l])
+        c.dispatch(self.x[l], T, self.idx[l], self.m, self.offsets[l], self.row_of[l], self.token_of[l],
+                   self.tile_expert[l], self.Xp[l])
+        c.expert_fwd(self.Xp[l], self.offsets[l], self.tile_expert[l], self.W_gu, self.W_down,
+                     self.base(l), self.m, self.GU[l], self.A[l], self.Yp[l])
+        c.combine(self.Yp[l], self.row_of[l], self.gate[l], T, self.x[l], self.x[l + 1])
+
+    def forward(self, x0=None, T=None):
+        T = self.T if T is None else T
+        if x0 is not None:
+            self.x[0, :T].copy_(x0, non_blocking=True)
+        for l in range(self.L):
+            self.forward_layer(l, T)
+        return self.x[self.L]
+
+    def aux_loss(self, T=None, fbar_prev=None):
+        T = self.T if T is None else T
+        c = self.ctx
+        if self.private:
+            for l in range(self.L):
+                c.pool_aux_loss(self.counts[l], self.score_sum[l], 1, self.m, T, self.alpha, None,
+                                self.loss[l:l + 1], self.coef[l], self.fbar[l])
+        else:
+            c.pool_aux_loss(self.counts, self.score_sum, self.L, self.m, T, self.alpha, fbar_prev,
+                            self.loss, self.coef[0], self.fbar[0])
+        return self.loss
+
+    # ------------------------------------------------------------------ backward
+    def backward_layer(self, l, dx_next, dx_out, T=None, with_aux=True):
+        T = self.T if T is None else T
+        c = self.ctx
+        s = l if self.deferred_wgrad else 0
+        flags = B.BWD_SKIP_WGRAD if self.deferred_wgrad else 0
+        c.expert_bwd(dx_next, T, self.row_of[l], self.gate[l], self.token_of[l], self.offsets[l],
+                     self.tile_expert[l], self.Xp[l], self.GU[l], self.A[l], self.Yp[l], self.W_gu,
+                     self.W_down, self.base(l), self.m, dx_next, self.dYp[s], self.dGU[s], dx_out,
+                     self.dgate, self.dW_gu, self.dW_down, flags)
+        coef = None
+        if with_aux:
+            coef = self.coef[l] if self.private else self.coef[0]
+        c.route_bwd(self.x[l], T, self.W_r[l], self.sigma[l], self.m, self.znorm[l], self.z[l],
+                    self.idx[l], self.dgate, coef, dx_out, self.dW_r[l], self.dsigma[l:l + 1])
+
+    def backward(self, upstream=None, T=None, with_aux=True):
+        T = self.T if T is None else T
+        cur = 0
+        if upstream is not None:
+            self.dx[cur, :T].copy_(upstream, non_blocking=True)
+        for l in reversed(range(self.L)):
+            self.backward_layer(l, self.dx[cur], self.dx[1 - cur], T, with_aux)
+            cur = 1 - cur
+        if self.deferred_wgrad:
+            self.ctx.pool_wgrad(self.L, self.cap, self.offsets, self.Xp, self.A, self.dYp, self.dGU,
+                                0, self.m, self.dW_gu, self.dW_down)
+        return self.dx[cur]
+
+    def step(self, x0=None, upstream=None, T=None):
+        """One pass of the whole hot path: forward, balance loss, backward."""
+        self.forward(x0, T)
+        self.aux_loss(T)
+        return self.backward(upstream, T)
+
+    def close(self):
+        self.ctx.close()

@@ -1,0 +1,285 @@
+"""GPU parity: every step of the CUDA path against the CPU oracle on the same
+seeded inputs, through the C-ABI (ctypes) binding.
+
+Tolerances (max|gpu - ref| / max|ref|): 1e-5 in fp32 mode, 1e-2 for bf16 storage
+with fp32 accumulation; balance loss relative 1e-5; routing indices, counts and
+the permutation maps bit-exact (indices: where the logit margin exceeds 1e-4).
+"""
+import numpy as np
+import pytest
+
+from oracle import unipool_oracle as O
+from paper_2605_06665_b200 import synth
+from parity_utils import (MARGIN, build_stack, calib_c, check_routing, f64, margin_safe, oracle_params,
+                          rel_max, to_np)
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"fp32": 1e-5, "bf16": 1e-2}
+
+
+def small_cfg(**kw):
+    cfg = dict(L=2, d=128, f=192, M=8, k=2, T=300, dtype="fp32", private=0, zipf_beta=0.0)
+    cfg.update(kw)
+    return cfg
+
+
+def run_layer_checks(cfg, T, L, seed=0, zero_grad_check=True):
+    """Runs the stack layer by layer; each layer's oracle consumes the GPU's own
+    x_l (and dx_{l+1}) so that only this layer's arithmetic is compared."""
+    import torch
+    inputs = synth.make_inputs(cfg, seed=seed, T=T, L=L)
+    st = build_stack(cfg, inputs, T=T, L=L)
+    tol = TOL[cfg["dtype"]]
+    k, m, M = cfg["k"], synth.router_width(cfg), cfg["M"]
+    pool, routers = oracle_params(inputs, L)
+    c, eps, alpha = st.c, synth.EPS, synth.ALPHA
+    st.x[0].copy_(torch.from_numpy(inputs["x0"]))
+    caches = []
+    for l in range(L):
+        st.forward_layer(l)
+        torch.cuda.synchronize()
+        x_l = f64(to_np(st.x[l]))
+        ref = O.route(x_l, routers[l]["W_r"], routers[l]["sigma"], c, eps, k, routers[l]["bias"])
+        idx_gpu = to_np(st.idx[l])
+        set_safe, order_safe = check_routing(idx_gpu, ref["z"], ref["idx"], k)
+        assert rel_max(to_np(st.z[l]), ref["z"]) < 1e-5
+        assert rel_max(to_np(st.znorm[l]), ref["n"]) < 1e-5
+        # everything downstream is compared with the GPU's own (valid) routing decision
+        ref = O.route(x_l, routers[l]["W_r"], routers[l]["sigma"], c, eps, k, routers[l]["bias"], forced_idx=idx_gpu)
+        assert rel_max(to_np(st.gate[l]), ref["g"]) < 1e-5
+        assert (to_np(st.counts[l]) == ref["counts"]).all()
+        assert to_np(st.counts[l]).sum() == T * k
+        assert rel_max(to_np(st.score_sum[l]), ref["S"]) < 1e-5
+        # permutation maps: bit-exact
+        off, row_of, token_of = O.dispatch_map(idx_gpu, m, 128)
+        assert (to_np(st.offsets[l]) == off).all()
+        assert (to_np(st.row_of[l]) == row_of).all()
+        used = int(off[-1])
+        tok_gpu = to_np(st.token_of[l])
+        assert (tok_gpu[:used] == token_of).all() and (tok_gpu[used:] == -1).all()
+        te = to_np(st.tile_expert[l])
+        exp_te = np.full(te.shape, -1)
+        for e in range(m):
+            exp_te[off[e] // 128:off[e + 1] // 128] = e
+        assert (te == exp_te).all()
+        Xp = to_np(st.Xp[l])[:used]
+        x_gpu = to_np(st.x[l])
+        assert (Xp[token_of >= 0] == x_gpu[token_of[token_of >= 0]]).all()      # pure data movement
+        assert not Xp[token_of < 0].any()
+        # expert FFN on the permuted rows
+        base = synth.expert_base(cfg, l)
+        GU, A, Yp = to_np(st.GU[l])[:used], to_np(st.A[l])[:used], to_np(st.Yp[l])[:used]
+        G_ref, U_ref, A_ref, Y_ref = (np.zeros((used, cfg["f"])), np.zeros((used, cfg["f"])),
+                                      np.zeros((used, cfg["f"])), np.zeros((used, cfg["d"])))
+        for e in range(m):
+            r0, r1 = int(off[e]), int(off[e + 1])
+            if r1 > r0:
+                G_ref[r0:r1], U_ref[r0:r1], A_ref[r0:r1], Y_ref[r0:r1] = O.expert_ffn(
+                    f64(Xp[r0:r1]), pool["W_gate"][base + e], pool["W_up"][base + e], pool["W_down"][base + e])
+        assert rel_max(GU[:, :cfg["f"]], G_ref) < tol and rel_max(GU[:, cfg["f"]:], U_ref) < tol
+        assert rel_max(A, A_ref) < tol and rel_max(Yp, Y_ref) < tol
+        assert not GU[token_of < 0].any() and not Yp[token_of < 0].any()        # pad rows stay zero
+        y_ref = O.moe_layer_output(x_l, idx_gpu, ref["g"], pool, base)
+        assert rel_max(to_np(st.x[l + 1]), x_l + y_ref) < tol
+        ref["x"] = x_l
+        caches.append(ref)
+    # balance loss
+    st.aux_loss()
+    torch.cuda.synchronize()
+    counts = np.stack([cc["counts"] for cc in caches])
+    S = np.stack([f64(to_np(st.score_sum[l])) for l in range(L)])
+    if cfg["private"]:
+        coefs = []
+        for l in range(L):
+            lo, fb, co = O.pool_aux_loss(counts[l:l + 1], S[l:l + 1], T, k, alpha)
+            assert abs(float(st.loss[l]) - lo) <= 1e-5 * abs(lo)
+            assert rel_max(to_np(st.coef[l]), co) < 1e-5
+            coefs.append(co)
+    else:
+        lo, fb, co = O.pool_aux_loss(counts, S, T, k, alpha)
+        assert abs(float(st.loss[0]) - lo) <= 1e-5 * abs(lo)
+        assert rel_max(to_np(st.coef[0]), co) < 1e-5 and rel_max(to_np(st.fbar[0]), fb) < 1e-5
+        coefs = [co] * L
+    # backward, layer by layer
+    st.zero_grad()
+    pool_grad = O.zeros_like_pool(pool)
+    dx_cur = torch.from_numpy(inputs["upstream"]).to(st.device, st.tdtype)
+    for l in reversed(range(L)):
+        dx_out = torch.empty_like(dx_cur)
+        st.backward_layer(l, dx_cur, dx_out)
+        torch.cuda.synchronize()
+        cc = caches[l]
+        base = synth.expert_base(cfg, l)
+        dxn = f64(to_np(dx_cur))
+        dx_e, dg = O.expert_path_backward(cc["x"], cc["idx"], cc["g"], pool, dxn, base, pool_grad)
+        assert rel_max(to_np(st.dgate), dg) < tol
+        rb = O.route_backward(cc["x"], routers[l]["W_r"], routers[l]["sigma"], c, eps, cc["z"], cc["n"],
+                              cc["idx"], dg, coefs[l])
+        assert rel_max(to_np(dx_out), dxn + dx_e + rb["dx"]) < tol
+        assert rel_max(to_np(st.dW_r[l]), rb["dW_r"]) < tol
+        assert abs(float(st.dsigma[l]) - rb["dsigma"]) <= tol * max(abs(rb["dsigma"]), 1e-3)
+        dx_cur = dx_out
+    f = cfg["f"]
+    dW_gu = to_np(st.dW_gu)
+    assert rel_max(dW_gu[:, :f], pool_grad["W_gate"]) < tol
+    assert rel_max(dW_gu[:, f:], pool_grad["W_up"]) < tol
+    assert rel_max(to_np(st.dW_down), pool_grad["W_down"]) < tol
+    if zero_grad_check:
+        used_experts = np.unique(np.concatenate(
+            [synth.expert_base(cfg, l) + cc["idx"].reshape(-1) for l, cc in enumerate(caches)]))
+        unused = np.setdiff1d(np.arange(M), used_experts)
+        assert not dW_gu[unused].any() and not to_np(st.dW_down)[unused].any()
+    st.ctx.check_status()
+    st.close()
+
+
+def test_tiny_fp32_layers():
+    cfg = synth.CONFIGS["tiny_fp32"]
+    run_layer_checks(cfg, cfg["T"], cfg["L"])
+
+
+@pytest.mark.parametrize("kw,T", [
+    (dict(), 300),                                   # ragged T, two tiles per group at most
+    (dict(M=5, k=1), 77),                            # k = 1, M not a multiple of anything
+    (dict(M=40, k=8, d=64, f=64), 130),              # k = 8
+    (dict(M=12, k=2, private=4, L=3), 200),          # layer-private layout (Eq. 1)
+    (dict(M=33, k=3), 1),                            # a single token: most experts empty
+    (dict(M=8, k=2, zipf_beta=3.0), 700),            # one giant group, several empty experts
+])
+def test_small_fp32_shapes(kw, T):
+    cfg = small_cfg(**kw)
+    run_layer_checks(cfg, T, cfg["L"], seed=3)
+
+
+@pytest.mark.parametrize("kw,T", [
+    (dict(dtype="bf16", d=256, f=384, M=16, k=2), 1000),
+    (dict(dtype="bf16", d=128, f=128, M=384, k=8, zipf_beta=0.35), 600),
+    (dict(dtype="bf16", d=256, f=256, M=12, k=2, private=4, L=3), 520),
+])
+def test_small_bf16_shapes(kw, T):
+    cfg = small_cfg(**kw)
+    run_layer_checks(cfg, T, cfg["L"], seed=4)
+
+
+def test_tiny_fp32_end_to_end():
+    """Config 1 without teacher forcing: forward, balance loss and backward of the
+    whole 4-layer stack against the float64 oracle."""
+    import torch
+    cfg = synth.CONFIGS["tiny_fp32"]
+    inputs = synth.make_inputs(cfg, seed=0)
+    st = build_stack(cfg, inputs)
+    L, T, k = cfg["L"], cfg["T"], cfg["k"]
+    pool, routers = oracle_params(inputs, L)
+    x0 = torch.from_numpy(inputs["x0"]).cuda()
+    up = torch.from_numpy(inputs["upstream"]).cuda()
+    st.zero_grad()
+    dx0 = st.step(x0, up)
+    torch.cuda.synchronize()
+    idx_gpu = [to_np(st.idx[l]) for l in range(L)]
+    free = O.stack_forward(f64(inputs["x0"]), routers, pool, k, st.c, synth.EPS)
+    for l in range(L):
+        check_routing(idx_gpu[l], free[l]["z"], free[l]["idx"], k)
+    res = O.stack_objective_and_grads(f64(inputs["x0"]), routers, pool, k, st.c, synth.EPS, synth.ALPHA,
+                                      f64(inputs["upstream"]), forced_idx=idx_gpu)
+    assert rel_max(to_np(st.x[L]), res["caches"][-1]["x_next"]) < 1e-5
+    assert abs(float(st.loss[0]) - res["loss_aux"]) <= 1e-5 * abs(res["loss_aux"])
+    f = cfg["f"]
+    assert rel_max(to_np(st.dW_gu)[:, :f], res["pool_grad"]["W_gate"]) < 1e-5
+    assert rel_max(to_np(st.dW_gu)[:, f:], res["pool_grad"]["W_up"]) < 1e-5
+    assert rel_max(to_np(st.dW_down), res["pool_grad"]["W_down"]) < 1e-5
+    for l in range(L):
+        assert rel_max(to_np(st.dW_r[l]), res["router_grads"][l]["dW_r"]) < 1e-5
+        assert abs(float(st.dsigma[l]) - res["router_grads"][l]["dsigma"]) <= 1e-5 * max(
+            1e-3, abs(res["router_grads"][l]["dsigma"]))
+    assert rel_max(to_np(dx0), res["dx0"]) < 1e-5
+    # determinism: a second pass gives bit-identical outputs and twice the gradients
+    xL_1 = st.x[L].clone()
+    g1 = st.dW_down.clone()
+    st.step(x0, up)
+    torch.cuda.synchronize()
+    assert torch.equal(xL_1, st.x[L])
+    assert rel_max(to_np(st.dW_down), 2 * to_np(g1)) < 1e-6
+    st.close()
+
+
+def test_empty_batch():
+    import torch
+    cfg = small_cfg()
+    inputs = synth.make_inputs(cfg, seed=1)
+    st = build_stack(cfg, inputs)
+    st.counts.fill_(7)
+    st.offsets.fill_(7)
+    st.zero_grad()
+    st.forward(T=0)
+    st.aux_loss(T=1)
+    st.backward(T=0)
+    torch.cuda.synchronize()
+    assert not to_np(st.counts).any() and not to_np(st.offsets).any()
+    assert not to_np(st.dW_gu).any()
+    st.ctx.check_status()
+    st.close()
+
+
+def test_deferred_pool_wgrad_matches_per_layer_accumulation():
+    import torch
+    cfg = small_cfg(dtype="bf16", d=256, f=384, M=16, k=2, L=3)
+    inputs = synth.make_inputs(cfg, seed=5, T=900)
+    x0 = torch.from_numpy(inputs["x0"]).cuda().bfloat16()
+    up = torch.from_numpy(inputs["upstream"]).cuda().bfloat16()
+    grads = []
+    for deferred in (False, True):
+        st = build_stack(cfg, inputs, T=900, deferred_wgrad=deferred)
+        st.zero_grad()
+        st.step(x0, up)
+        torch.cuda.synchronize()
+        grads.append((to_np(st.dW_gu), to_np(st.dW_down)))
+        st.close()
+    assert rel_max(grads[1][0], grads[0][0]) < 1e-5
+    assert rel_max(grads[1][1], grads[0][1]) < 1e-5
+
+
+def test_one_step_behind_fbar():
+    import torch
+    cfg = small_cfg(M=8)
+    inputs = synth.make_inputs(cfg, seed=6)
+    st = build_stack(cfg, inputs)
+    st.forward(torch.from_numpy(inputs["x0"]).cuda())
+    prev = np.random.default_rng(0).dirichlet(np.ones(8)).astype(np.float32)
+    st.aux_loss(fbar_prev=torch.from_numpy(prev).cuda())
+    torch.cuda.synchronize()
+    lo, fb, co = O.pool_aux_loss(to_np(st.counts).astype(np.int64), f64(to_np(st.score_sum)), cfg["T"], cfg["k"],
+                                 synth.ALPHA, fbar_prev=f64(prev))
+    assert abs(float(st.loss[0]) - lo) <= 1e-5 * abs(lo)
+    assert rel_max(to_np(st.coef[0]), co) < 1e-5 and rel_max(to_np(st.fbar[0]), fb) < 1e-5
+    st.close()
+
+
+def test_calibrate_c_on_device():
+    from oracle import norm_router_c
+    cfg = small_cfg()
+    st = build_stack(cfg, synth.make_inputs(cfg, seed=0))
+    for (E, k) in [(96, 2), (16, 2), (384, 8)]:
+        got = st.ctx.calibrate_c(E, k, 200_000, seed=1)
+        ref = norm_router_c.estimate_c(E, k, 200_000, seed=2)
+        assert got >= 1.0 and abs(got - ref) / ref < 5e-3
+    st.close()
+
+
+def test_corrupt_routing_table_is_reported_not_faulted():
+    """An out-of-range expert id is caught by the dispatch kernel's own bounds check:
+    the assignment is dropped and the status word reports it."""
+    import torch
+    from paper_2605_06665_b200 import binding as B
+    cfg = small_cfg()
+    st = build_stack(cfg, synth.make_inputs(cfg, seed=0))
+    st.forward_layer(0)
+    st.idx[0, 5, 1] = 1000
+    st.ctx.dispatch(st.x[0], cfg["T"], st.idx[0], cfg["M"], st.offsets[0], st.row_of[0], st.token_of[0],
+                    st.tile_expert[0], st.Xp[0])
+    with pytest.raises(B.UniPoolError) as ei:
+        st.ctx.check_status()
+    assert ei.value.code == -6
+    assert int(st.row_of[0, 5, 1]) == -1
+    st.ctx.check_status()          # cleared
+    st.close()
