@@ -2,6 +2,7 @@
 // Every compute step is a CUDA kernel in one of the other translation units.
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 
@@ -16,6 +17,13 @@ void set_error(const char* fmt, ...) {
   va_start(ap, fmt);
   vsnprintf(g_error, sizeof(g_error), fmt, ap);
   va_end(ap);
+}
+
+// Debug aid: UNIPOOL_FORCE_SIMT=1 runs the bf16 grouped GEMMs on the CUDA-core path
+// (same arithmetic contract, far slower); used to bisect tensor-core issues.
+static bool use_tensor_cores(const unipool_ctx* ctx) {
+  static const bool forced = [] { const char* v = getenv("UNIPOOL_FORCE_SIMT"); return v && v[0] == '1'; }();
+  return ctx->cfg.dtype == UNIPOOL_BF16 && !forced;
 }
 
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -194,7 +202,7 @@ int unipool_expert_fwd(unipool_ctx* ctx, const void* Xp, const int32_t* offsets,
   CHECK_PTR(GU); CHECK_PTR(A); CHECK_PTR(Yp);
   ExpertFwdArgs a{Xp, offsets, tile_expert, W_gu, W_down, expert_base, n_experts, GU, A, Yp};
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  return ctx->cfg.dtype == UNIPOOL_BF16 ? expert_fwd_tc(ctx, a, s) : expert_fwd_simt(ctx, a, s);
+  return use_tensor_cores(ctx) ? expert_fwd_tc(ctx, a, s) : expert_fwd_simt(ctx, a, s);
 }
 
 int unipool_combine(unipool_ctx* ctx, const void* Yp, const int32_t* row_of, const float* gate,
@@ -223,7 +231,7 @@ int unipool_expert_bwd(unipool_ctx* ctx, const void* dy, int32_t T, const int32_
   if (rc != UNIPOOL_OK) return rc;
   ExpertBwdArgs a{offsets, tile_expert, Xp, GU, A, W_gu, W_down, expert_base, n_experts,
                   dYp, dGU, ctx->ws.dXp, dW_gu, dW_down, wgrad};
-  rc = ctx->cfg.dtype == UNIPOOL_BF16 ? expert_bwd_tc(ctx, a, s) : expert_bwd_simt(ctx, a, s);
+  rc = use_tensor_cores(ctx) ? expert_bwd_tc(ctx, a, s) : expert_bwd_simt(ctx, a, s);
   if (rc != UNIPOOL_OK) return rc;
   return unpermute_sum_launch(ctx, ctx->ws.dXp, row_of, T, dx_residual, dx, s);
 }
@@ -241,7 +249,7 @@ int unipool_pool_wgrad(unipool_ctx* ctx, int32_t n_layers, int64_t layer_stride_
   PoolWgradArgs a{n_layers, layer_stride_rows, offsets, Xp, A, dYp, dGU, expert_base, n_experts,
                   dW_gu, dW_down};
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  return ctx->cfg.dtype == UNIPOOL_BF16 ? pool_wgrad_tc(ctx, a, s) : pool_wgrad_simt(ctx, a, s);
+  return use_tensor_cores(ctx) ? pool_wgrad_tc(ctx, a, s) : pool_wgrad_simt(ctx, a, s);
 }
 
 int unipool_pool_aux_loss(unipool_ctx* ctx, const int32_t* counts, const float* score_sum,

@@ -1,9 +1,541 @@
-// placeholder: tensor-core grouped GEMMs land here; bring-up routes to the CUDA-core path.
+// Grouped SwiGLU expert GEMMs on the 5th-generation tensor cores (tcgen05) for
+// bf16 storage with fp32 accumulation: forward (Eq. 2's e_i), dgrad and wgrad.
+//
+// One persistent, warp-specialised kernel template serves all six GEMMs:
+//   warp 0      TMA producer   (one lane issues cp.async.bulk.tensor loads)
+//   warp 1      MMA issuer     (one lane issues tcgen05.mma; owns the TMEM allocation)
+//   warps 2-5   epilogue       (tcgen05.ld from TMEM, fused element-wise math, global stores)
+// Operand tiles are staged in shared memory with the 128-byte swizzle, accumulators
+// are double-buffered in TMEM so the epilogue of one tile overlaps the main loop of
+// the next.  The tile schedule is read from device memory (group offsets), so no call
+// synchronises the host.  Every mbarrier wait is bounded: on expiry the kernel records
+// UNIPOOL_ERR_TIMEOUT in the status word, all roles leave, TMEM is released.
+#include <cuda.h>
+
 #include "common.cuh"
+#include "tc_ptx.cuh"
+
 namespace unipool {
-int tc_module_init(unipool_ctx*) { return UNIPOOL_OK; }
-void tc_module_destroy(unipool_ctx*) {}
-int expert_fwd_tc(unipool_ctx* c, const ExpertFwdArgs& a, cudaStream_t s) { return expert_fwd_simt(c, a, s); }
-int expert_bwd_tc(unipool_ctx* c, const ExpertBwdArgs& a, cudaStream_t s) { return expert_bwd_simt(c, a, s); }
-int pool_wgrad_tc(unipool_ctx* c, const PoolWgradArgs& a, cudaStream_t s) { return pool_wgrad_simt(c, a, s); }
+
+namespace {
+
+constexpr int BM = 128;          // rows of an output tile (TMEM lanes)
+constexpr int BK = 64;           // k-block: 64 bf16 = one 128-byte swizzle row
+constexpr int kThreads = 192;
+constexpr uint32_t kABytes = BM * BK * 2;
+constexpr uint32_t kMnBlockBytes = 64 * BK * 2;   // one 64(MN) x 64(K) box
+
+enum Mode : int {
+  kFwd1 = 0,    // GU = Xp W_gu^T, A = silu(G)*U        A K-major, B K-major (3-D map), row tiles
+  kFwd2 = 1,    // Yp = A W_down^T                      A K-major, B K-major,           row tiles
+  kDgrad1 = 2,  // dGU = swiglu'(dYp W_down, GU)        A K-major, B MN-major,          row tiles
+  kDgrad2 = 3,  // dXp = dGU W_gu                       A K-major, B MN-major,          row tiles
+  kWgrad = 4,   // dW[e] += P_e^T Q_e                   A MN-major, B MN-major,         ragged K
+};
+
+struct GemmParams {
+  const int32_t* offsets;       // row tiles: &offsets[n_experts]; wgrad: [n_layers][n_experts+1]
+  const int32_t* tile_expert;   // row tiles only
+  int n_experts, expert_base;
+  int n_layers;                 // wgrad
+  int layer_stride_rows;        // wgrad
+  int Mdim, Ndim, Kdim;         // wgrad: dW is [Mdim, Ndim]; row tiles: output columns, contraction
+  int f;                        // expert width (fwd1 / dgrad1 addressing)
+  __nv_bfloat16* out0;          // fwd1: GU; fwd2: Yp; dgrad1: dGU; dgrad2: dXp
+  __nv_bfloat16* out1;          // fwd1: A
+  const __nv_bfloat16* GU;      // dgrad1
+  float* dW;                    // wgrad
+  int32_t* status;
+};
+
+template <int BN> struct SmemLayout {
+  static constexpr uint32_t kBBytes = BN * BK * 2;
+  static constexpr uint32_t kStageBytes = kABytes + kBBytes;
+  static constexpr int kStages = BN == 256 ? 4 : 6;
+  static constexpr uint32_t kBarOffset = kStages * kStageBytes;
+  static constexpr uint32_t kTotal = kBarOffset + 256 + 1024;   // + barriers + alignment slack
+};
+
+template <int MODE> struct Traits {
+  static constexpr bool kAMn = MODE == kWgrad;
+  static constexpr bool kBMn = MODE == kDgrad1 || MODE == kDgrad2 || MODE == kWgrad;
+  static constexpr bool kRowTiles = MODE != kWgrad;
+};
+
+struct TileCoord { int e, mt, nt, kblocks; bool valid; };
+
+template <int MODE, int BN>
+__device__ __forceinline__ int tiles_total(const GemmParams& p, int& n_nt, int& n_mt) {
+  if constexpr (Traits<MODE>::kRowTiles) {
+    n_mt = *p.offsets / BM;
+    const int ncols = MODE == kFwd1 ? BN / 2 : BN;
+    n_nt = (p.Ndim + ncols - 1) / ncols;
+    return n_mt * n_nt;
+  } else {
+    n_mt = (p.Mdim + BM - 1) / BM;
+    n_nt = (p.Ndim + BN - 1) / BN;
+    return p.n_experts * n_mt * n_nt;
+  }
 }
+
+template <int MODE>
+__device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int tile, int n_nt, int n_mt) {
+  TileCoord c;
+  if constexpr (Traits<MODE>::kRowTiles) {
+    c.mt = tile / n_nt;
+    c.nt = tile % n_nt;
+    c.e = p.tile_expert[c.mt];
+    c.kblocks = p.Kdim / BK;
+    c.valid = c.e >= 0 && c.e < p.n_experts;
+  } else {
+    const int per_e = n_mt * n_nt;
+    c.e = tile / per_e;
+    const int rem = tile % per_e;
+    c.mt = rem / n_nt;
+    c.nt = rem % n_nt;
+    int kb = 0;
+    for (int l = 0; l < p.n_layers; ++l) {
+      const int32_t* off = p.offsets + (int64_t)l * (p.n_experts + 1);
+      kb += (off[c.e + 1] - off[c.e]) / BK;
+    }
+    c.kblocks = kb;
+    c.valid = kb > 0;
+  }
+  return c;
+}
+
+__device__ __forceinline__ void report_timeout(const GemmParams& p, volatile int* abort, int site) {
+  *abort = 1;
+  if (atomicCAS(p.status, 0, kStatusTimeout) == 0) {
+    p.status[1] = site;
+    p.status[2] = (int)blockIdx.x;
+  }
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// 32 consecutive bf16 of one row -> global (64 bytes, four 16-byte stores)
+__device__ __forceinline__ void store_row32(__nv_bfloat16* dst, const float (&v)[32]) {
+  uint4* d4 = reinterpret_cast<uint4*>(dst);
+#pragma unroll
+  for (int q = 0; q < 4; ++q)
+    d4[q] = make_uint4(pack_bf16(v[8 * q + 0], v[8 * q + 1]), pack_bf16(v[8 * q + 2], v[8 * q + 3]),
+                       pack_bf16(v[8 * q + 4], v[8 * q + 5]), pack_bf16(v[8 * q + 6], v[8 * q + 7]));
+}
+__device__ __forceinline__ void load_row32(const __nv_bfloat16* src, float (&v)[32]) {
+  const uint4* s4 = reinterpret_cast<const uint4*>(src);
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const uint4 w = __ldg(s4 + q);
+    const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      v[8 * q + 2 * i] = __uint_as_float(ww[i] << 16);
+      v[8 * q + 2 * i + 1] = __uint_as_float(ww[i] & 0xffff0000u);
+    }
+  }
+}
+
+template <int MODE, int BN>
+__global__ void __launch_bounds__(kThreads, 1)
+grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                       const GemmParams p) {
+  using L = SmemLayout<BN>;
+  using TR = Traits<MODE>;
+  constexpr int kStages = L::kStages;
+  constexpr uint32_t kTmemCols = 2 * BN;            // two accumulators of BN fp32 columns
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + L::kBarOffset);
+  uint64_t* empty_bar = full_bar + kStages;
+  uint64_t* tmem_full = empty_bar + kStages;
+  uint64_t* tmem_empty = tmem_full + 2;
+  uint32_t* tmem_ptr = reinterpret_cast<uint32_t*>(tmem_empty + 2);
+  volatile int* abort = reinterpret_cast<volatile int*>(tmem_ptr + 1);
+
+  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) { tc::mbar_init(&full_bar[s], 1); tc::mbar_init(&empty_bar[s], 1); }
+    for (int a = 0; a < 2; ++a) { tc::mbar_init(&tmem_full[a], 1); tc::mbar_init(&tmem_empty[a], 4); }
+    *abort = 0;
+    tc::fence_barrier_init();
+    tc::tma_prefetch_desc(&tmA);
+    tc::tma_prefetch_desc(&tmB);
+  }
+  if (warp == 1) {
+    tc::tmem_alloc(tmem_ptr, kTmemCols);
+    tc::tmem_relinquish();
+  }
+  tc::tc_fence_before_sync();
+  __syncthreads();
+  tc::tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_ptr;
+
+  int n_nt, n_mt;
+  const int total = tiles_total<MODE, BN>(p, n_nt, n_mt);
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
+        const TileCoord c = tile_coord<MODE>(p, tile, n_nt, n_mt);
+        if (!c.valid) continue;
+        const int pe = p.expert_base + c.e;
+        int layer = 0, r = 0, r_end = 0;              // wgrad: walks the rows of expert e, layer by layer
+        if constexpr (!TR::kRowTiles) {
+          r = p.offsets[c.e];
+          r_end = p.offsets[c.e + 1];
+        }
+        for (int kb = 0; kb < c.kblocks; ++kb) {
+          if (!tc::mbar_wait(&empty_bar[stage], phase ^ 1u, abort)) { report_timeout(p, abort, 1); ok = false; break; }
+          uint8_t* sA = smem + stage * L::kStageBytes;
+          uint8_t* sB = sA + kABytes;
+          tc::mbar_expect_tx(&full_bar[stage], L::kStageBytes);
+          if constexpr (MODE == kFwd1) {
+            tc::tma_load_2d(sA, &tmA, &full_bar[stage], kb * BK, c.mt * BM);
+            tc::tma_load_3d(sB, &tmB, &full_bar[stage], kb * BK, c.nt * (BN / 2), 2 * pe);
+          } else if constexpr (MODE == kFwd2) {
+            tc::tma_load_2d(sA, &tmA, &full_bar[stage], kb * BK, c.mt * BM);
+            tc::tma_load_2d(sB, &tmB, &full_bar[stage], kb * BK, pe * p.Ndim + c.nt * BN);
+          } else if constexpr (MODE == kDgrad1 || MODE == kDgrad2) {
+            tc::tma_load_2d(sA, &tmA, &full_bar[stage], kb * BK, c.mt * BM);
+#pragma unroll
+            for (int i = 0; i < BN / 64; ++i)
+              tc::tma_load_2d(sB + i * kMnBlockBytes, &tmB, &full_bar[stage], c.nt * BN + 64 * i,
+                              pe * p.Kdim + kb * BK);
+          } else {
+            while (r >= r_end) {                        // next layer that has rows for this expert
+              ++layer;
+              const int32_t* off = p.offsets + (int64_t)layer * (p.n_experts + 1);
+              r = off[c.e];
+              r_end = off[c.e + 1];
+            }
+            const int grow = layer * p.layer_stride_rows + r;
+#pragma unroll
+            for (int i = 0; i < BM / 64; ++i)
+              tc::tma_load_2d(sA + i * kMnBlockBytes, &tmA, &full_bar[stage], c.mt * BM + 64 * i, grow);
+#pragma unroll
+            for (int i = 0; i < BN / 64; ++i)
+              tc::tma_load_2d(sB + i * kMnBlockBytes, &tmB, &full_bar[stage], c.nt * BN + 64 * i, grow);
+            r += BK;
+          }
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {
+        // give loads already in flight time to land before the CTA retires
+        for (int i = 0; i < 200; ++i) __nanosleep(1000);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = tc::instr_desc_bf16(BN, TR::kAMn, TR::kBMn);
+      constexpr uint32_t a_lbo = TR::kAMn ? kMnBlockBytes : 16, b_lbo = TR::kBMn ? kMnBlockBytes : 16;
+      constexpr uint32_t a_step = (TR::kAMn ? 16 * 128 : 32) >> 4;   // descriptor units of 16 bytes per K = 16
+      constexpr uint32_t b_step = (TR::kBMn ? 16 * 128 : 32) >> 4;
+      int stage = 0;
+      uint32_t phase = 0;
+      int local = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
+        const TileCoord c = tile_coord<MODE>(p, tile, n_nt, n_mt);
+        if (!c.valid) continue;
+        const int acc = local & 1;
+        const uint32_t acc_phase = (local >> 1) & 1;
+        ++local;
+        if (!tc::mbar_wait(&tmem_empty[acc], acc_phase ^ 1u, abort)) { report_timeout(p, abort, 2); break; }
+        tc::tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + acc * BN;
+        for (int kb = 0; kb < c.kblocks; ++kb) {
+          if (!tc::mbar_wait(&full_bar[stage], phase, abort)) { report_timeout(p, abort, 3); ok = false; break; }
+          tc::tc_fence_after_sync();
+          const uint32_t aaddr = tc::smem_u32(smem + stage * L::kStageBytes);
+          const uint64_t adesc = tc::smem_desc_sw128(aaddr, a_lbo, 1024);
+          const uint64_t bdesc = tc::smem_desc_sw128(aaddr + kABytes, b_lbo, 1024);
+#pragma unroll
+          for (int j = 0; j < BK / 16; ++j)
+            tc::umma_bf16(d_tmem, adesc + j * a_step, bdesc + j * b_step, idesc, (kb | j) != 0 ? 1u : 0u);
+          tc::umma_commit(&empty_bar[stage]);            // frees the stage once these MMAs have read it
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (ok) tc::umma_commit(&tmem_full[acc]);        // accumulator complete
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue (warps 2..5)
+    const int quarter = warp & 3;                        // TMEM lanes [32*quarter, 32*quarter + 32)
+    int local = 0;
+    for (int tile = blockIdx.x; tile < total; tile += gridDim.x) {
+      const TileCoord c = tile_coord<MODE>(p, tile, n_nt, n_mt);
+      if (!c.valid) continue;
+      const int acc = local & 1;
+      const uint32_t acc_phase = (local >> 1) & 1;
+      ++local;
+      if (!tc::mbar_wait(&tmem_full[acc], acc_phase, abort)) {
+        if (lane == 0) report_timeout(p, abort, 4);
+        break;
+      }
+      tc::tc_fence_after_sync();
+      const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * BN;
+      const int row_in_tile = quarter * 32 + lane;
+
+      if constexpr (MODE == kFwd1) {
+        const int64_t row = (int64_t)c.mt * BM + row_in_tile;
+        const int feat0 = c.nt * (BN / 2);
+#pragma unroll 1
+        for (int ch = 0; ch < BN / 64; ++ch) {
+          uint32_t rg[32], ru[32];
+          tc::tmem_ld_32x32(t_row + ch * 32, rg);
+          tc::tmem_ld_32x32(t_row + BN / 2 + ch * 32, ru);
+          tc::tmem_ld_wait();
+          const int feat = feat0 + ch * 32;
+          if (feat < p.f) {
+            float g[32], u[32], a[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              g[i] = __uint_as_float(rg[i]);
+              u[i] = __uint_as_float(ru[i]);
+              a[i] = silu_f(g[i]) * u[i];
+            }
+            store_row32(p.out0 + row * 2 * p.f + feat, g);
+            store_row32(p.out0 + row * 2 * p.f + p.f + feat, u);
+            store_row32(p.out1 + row * p.f + feat, a);
+          }
+        }
+      } else if constexpr (MODE == kFwd2 || MODE == kDgrad2) {
+        const int64_t row = (int64_t)c.mt * BM + row_in_tile;
+#pragma unroll 1
+        for (int ch = 0; ch < BN / 32; ++ch) {
+          uint32_t rr[32];
+          tc::tmem_ld_32x32(t_row + ch * 32, rr);
+          tc::tmem_ld_wait();
+          const int col = c.nt * BN + ch * 32;
+          if (col < p.Ndim) {
+            float v[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(rr[i]);
+            store_row32(p.out0 + row * p.Ndim + col, v);
+          }
+        }
+      } else if constexpr (MODE == kDgrad1) {
+        const int64_t row = (int64_t)c.mt * BM + row_in_tile;
+#pragma unroll 1
+        for (int ch = 0; ch < BN / 32; ++ch) {
+          uint32_t rr[32];
+          tc::tmem_ld_32x32(t_row + ch * 32, rr);
+          tc::tmem_ld_wait();
+          const int col = c.nt * BN + ch * 32;
+          if (col < p.f) {
+            float g[32], u[32], dg[32], du[32];
+            load_row32(p.GU + row * 2 * p.f + col, g);
+            load_row32(p.GU + row * 2 * p.f + p.f + col, u);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const float dA = __uint_as_float(rr[i]);
+              dg[i] = dA * u[i] * silu_grad_f(g[i]);
+              du[i] = dA * silu_f(g[i]);
+            }
+            store_row32(p.out0 + row * 2 * p.f + col, dg);
+            store_row32(p.out0 + row * 2 * p.f + p.f + col, du);
+          }
+        }
+      } else {
+        const int m = c.mt * BM + row_in_tile;
+        float* out = p.dW + ((int64_t)(p.expert_base + c.e) * p.Mdim + m) * p.Ndim;
+#pragma unroll 1
+        for (int ch = 0; ch < BN / 32; ++ch) {
+          uint32_t rr[32];
+          tc::tmem_ld_32x32(t_row + ch * 32, rr);
+          tc::tmem_ld_wait();
+          const int col = c.nt * BN + ch * 32;
+          if (m < p.Mdim && col < p.Ndim) {
+            float4* o4 = reinterpret_cast<float4*>(out + col);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+              float4 cur = o4[q];
+              cur.x += __uint_as_float(rr[4 * q + 0]);
+              cur.y += __uint_as_float(rr[4 * q + 1]);
+              cur.z += __uint_as_float(rr[4 * q + 2]);
+              cur.w += __uint_as_float(rr[4 * q + 3]);
+              o4[q] = cur;
+            }
+          }
+        }
+      }
+      tc::tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) tc::mbar_arrive(&tmem_empty[acc]);
+    }
+  }
+
+  tc::tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    tc::tc_fence_after_sync();
+    tc::tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// ---------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct TcModule {
+  EncodeTiledFn encode;
+};
+
+// bf16 tensor map with the 128-byte swizzle; dims/box innermost first, strides in elements.
+int make_tmap(const unipool_ctx* ctx, CUtensorMap* out, const void* base, int rank, const uint64_t* dims,
+              const uint64_t* strides_elems, const uint32_t* box) {
+  const TcModule* mod = static_cast<const TcModule*>(ctx->tmap_cache);
+  cuuint64_t gdims[3], gstrides[2];
+  cuuint32_t gbox[3], estr[3] = {1, 1, 1};
+  for (int i = 0; i < rank; ++i) { gdims[i] = dims[i]; gbox[i] = box[i]; }
+  for (int i = 0; i + 1 < rank; ++i) gstrides[i] = strides_elems[i] * 2;
+  UP_REQUIRE((reinterpret_cast<uintptr_t>(base) & 15) == 0, UNIPOOL_ERR_INVALID_ARG,
+             "tensor base %p is not 16-byte aligned", base);
+  CUresult r = mod->encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gdims,
+                           gstrides, gbox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  UP_REQUIRE(r == CUDA_SUCCESS, UNIPOOL_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+  return UNIPOOL_OK;
+}
+
+int map_2d(const unipool_ctx* ctx, CUtensorMap* out, const void* base, uint64_t cols, uint64_t rows,
+           uint32_t box_cols, uint32_t box_rows) {
+  const uint64_t dims[2] = {cols, rows}, strides[1] = {cols};
+  const uint32_t box[2] = {box_cols, box_rows};
+  return make_tmap(ctx, out, base, 2, dims, strides, box);
+}
+
+template <int MODE, int BN>
+int launch(unipool_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmParams& p, cudaStream_t s) {
+  auto kern = grouped_gemm_tc_kernel<MODE, BN>;
+  constexpr int smem = SmemLayout<BN>::kTotal;
+  UP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+  kern<<<ctx->sm_count, kThreads, smem, s>>>(tmA, tmB, p);
+  UP_LAUNCH_CHECK();
+  return UNIPOOL_OK;
+}
+
+int wgrad_pair(unipool_ctx* ctx, const PoolWgradArgs& a, cudaStream_t s) {
+  const int d = ctx->cfg.d_model, f = ctx->cfg.d_ff;
+  const uint64_t rows = (uint64_t)(a.n_layers > 1 ? (int64_t)a.n_layers * a.layer_stride_rows : ctx->row_capacity);
+  GemmParams p{};
+  p.offsets = a.offsets;
+  p.n_experts = a.n_experts;
+  p.expert_base = a.expert_base;
+  p.n_layers = a.n_layers;
+  p.layer_stride_rows = (int)a.layer_stride_rows;
+  p.status = ctx->ws.status;
+  CUtensorMap tmP, tmQ;
+  int rc;
+  // dW_down[e] [d, f] += dYp_e^T A_e
+  if ((rc = map_2d(ctx, &tmP, a.dYp, d, rows, 64, 64)) != UNIPOOL_OK) return rc;
+  if ((rc = map_2d(ctx, &tmQ, a.A, f, rows, 64, 64)) != UNIPOOL_OK) return rc;
+  p.Mdim = d; p.Ndim = f; p.dW = a.dW_down;
+  if ((rc = launch<kWgrad, 128>(ctx, tmP, tmQ, p, s)) != UNIPOOL_OK) return rc;
+  // dW_gu[e] [2f, d] += dGU_e^T Xp_e
+  if ((rc = map_2d(ctx, &tmP, a.dGU, 2 * f, rows, 64, 64)) != UNIPOOL_OK) return rc;
+  if ((rc = map_2d(ctx, &tmQ, a.Xp, d, rows, 64, 64)) != UNIPOOL_OK) return rc;
+  p.Mdim = 2 * f; p.Ndim = d; p.dW = a.dW_gu;
+  return launch<kWgrad, 128>(ctx, tmP, tmQ, p, s);
+}
+
+}  // namespace
+
+int tc_module_init(unipool_ctx* ctx) {
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
+  UP_REQUIRE(e == cudaSuccess && fn != nullptr && q == cudaDriverEntryPointSuccess, UNIPOOL_ERR_CUDA,
+             "cuTensorMapEncodeTiled is not available from the driver (%s)", cudaGetErrorString(e));
+  TcModule* mod = new TcModule{reinterpret_cast<EncodeTiledFn>(fn)};
+  ctx->tmap_cache = mod;
+  return UNIPOOL_OK;
+}
+
+void tc_module_destroy(unipool_ctx* ctx) {
+  delete static_cast<TcModule*>(ctx->tmap_cache);
+  ctx->tmap_cache = nullptr;
+}
+
+int expert_fwd_tc(unipool_ctx* ctx, const ExpertFwdArgs& a, cudaStream_t s) {
+  const int d = ctx->cfg.d_model, f = ctx->cfg.d_ff, M = ctx->cfg.pool_size;
+  const uint64_t cap = (uint64_t)ctx->row_capacity;
+  GemmParams p{};
+  p.offsets = a.offsets + a.n_experts;
+  p.tile_expert = a.tile_expert;
+  p.n_experts = a.n_experts;
+  p.expert_base = a.expert_base;
+  p.f = f;
+  p.status = ctx->ws.status;
+  CUtensorMap tmA, tmB;
+  int rc;
+  // GU = Xp [W_gate; W_up]^T with the SwiGLU epilogue.  B tile = 64 gate rows + 64 up rows of the
+  // same features, fetched as one 3-D box over W_gu viewed as [2M, f, d].
+  if ((rc = map_2d(ctx, &tmA, a.Xp, d, cap, 64, 128)) != UNIPOOL_OK) return rc;
+  {
+    const uint64_t dims[3] = {(uint64_t)d, (uint64_t)f, (uint64_t)2 * M};
+    const uint64_t strides[2] = {(uint64_t)d, (uint64_t)f * d};
+    const uint32_t box[3] = {64, 64, 2};
+    if ((rc = make_tmap(ctx, &tmB, a.W_gu, 3, dims, strides, box)) != UNIPOOL_OK) return rc;
+  }
+  p.Ndim = f; p.Kdim = d;
+  p.out0 = static_cast<__nv_bfloat16*>(a.GU);
+  p.out1 = static_cast<__nv_bfloat16*>(a.A);
+  if ((rc = launch<kFwd1, 128>(ctx, tmA, tmB, p, s)) != UNIPOOL_OK) return rc;
+  // Yp = A W_down^T
+  if ((rc = map_2d(ctx, &tmA, a.A, f, cap, 64, 128)) != UNIPOOL_OK) return rc;
+  if ((rc = map_2d(ctx, &tmB, a.W_down, f, (uint64_t)M * d, 64, 128)) != UNIPOOL_OK) return rc;
+  p.Ndim = d; p.Kdim = f;
+  p.out0 = static_cast<__nv_bfloat16*>(a.Yp);
+  p.out1 = nullptr;
+  return launch<kFwd2, 128>(ctx, tmA, tmB, p, s);
+}
+
+int expert_bwd_tc(unipool_ctx* ctx, const ExpertBwdArgs& a, cudaStream_t s) {
+  const int d = ctx->cfg.d_model, f = ctx->cfg.d_ff, M = ctx->cfg.pool_size;
+  const uint64_t cap = (uint64_t)ctx->row_capacity;
+  GemmParams p{};
+  p.offsets = a.offsets + a.n_experts;
+  p.tile_expert = a.tile_expert;
+  p.n_experts = a.n_experts;
+  p.expert_base = a.expert_base;
+  p.f = f;
+  p.status = ctx->ws.status;
+  CUtensorMap tmA, tmB;
+  int rc;
+  // dA = dYp W_down, fused with the SwiGLU derivative -> dGU
+  if ((rc = map_2d(ctx, &tmA, a.dYp, d, cap, 64, 128)) != UNIPOOL_OK) return rc;
+  if ((rc = map_2d(ctx, &tmB, a.W_down, f, (uint64_t)M * d, 64, 64)) != UNIPOOL_OK) return rc;
+  p.Ndim = f; p.Kdim = d;
+  p.GU = static_cast<const __nv_bfloat16*>(a.GU);
+  p.out0 = static_cast<__nv_bfloat16*>(a.dGU);
+  if ((rc = launch<kDgrad1, 128>(ctx, tmA, tmB, p, s)) != UNIPOOL_OK) return rc;
+  // dXp = dGU [W_gate; W_up]
+  if ((rc = map_2d(ctx, &tmA, a.dGU, 2 * f, cap, 64, 128)) != UNIPOOL_OK) return rc;
+  if ((rc = map_2d(ctx, &tmB, a.W_gu, d, (uint64_t)M * 2 * f, 64, 64)) != UNIPOOL_OK) return rc;
+  p.Ndim = d; p.Kdim = 2 * f;
+  p.out0 = static_cast<__nv_bfloat16*>(a.dXp);
+  if ((rc = launch<kDgrad2, 128>(ctx, tmA, tmB, p, s)) != UNIPOOL_OK) return rc;
+  if (a.wgrad) {
+    PoolWgradArgs w{1, 0, a.offsets, a.Xp, a.A, a.dYp, a.dGU, a.expert_base, a.n_experts, a.dW_gu, a.dW_down};
+    return wgrad_pair(ctx, w, s);
+  }
+  return UNIPOOL_OK;
+}
+
+int pool_wgrad_tc(unipool_ctx* ctx, const PoolWgradArgs& a, cudaStream_t s) { return wgrad_pair(ctx, a, s); }
+
+}  // namespace unipool
