@@ -1,0 +1,350 @@
+#!/usr/bin/env python
+"""Benchmark of the UniPool MoE-layer hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+A "step" is one pass of the whole hot path over one synthetic batch: for every
+layer route -> dispatch -> grouped expert FFN -> combine, then the pool balance
+loss, then for every layer (in reverse) expert backward (dgrad + wgrad into the
+shared fp32 pool gradient) and router backward.  The metric is MoE-layer
+fwd+bwd tokens per second: tokens * layers / step time, summed over all GPUs
+(each rank runs the same workload on its own token shard; no data-path
+collective - the layer is token-parallel).
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle, as it
+stands, on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "moe_layer_fwd_bwd_tokens_per_s"
+UNIT = "tokens/s"
+
+# algorithmic FLOPs of the grouped GEMM phases per routed row: 2*d*f per (row, GEMM of d x f)
+GEMM_PHASES = {"expert_fwd_gu": 4, "expert_fwd_down": 2, "dgrad_down": 2, "dgrad_gu": 4, "wgrad_down": 2,
+               "wgrad_gu": 4}
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_tflops=p["bf16_tflops"],
+                    bf16_tflops_sustained=p.get("bf16_tflops_sustained", p["bf16_tflops"]), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu_index), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "200"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        time.sleep(0.25)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1])); smax.append(float(parts[2])); power.append(float(parts[3]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        sm.sort()
+        return dict(sm_mhz=sm[len(sm) // 2] if sm else None, sm_max_mhz=max(smax) if smax else None,
+                    power_w_max=max(power) if power else None, samples=len(sm), reasons=sorted(reasons))
+
+
+def algorithmic_bytes(cfg, cap_rows):
+    """HBM bytes the memory-bound phases must move per launch (bf16 activations)."""
+    T, d, k, m = cfg["T"], cfg["d"], cfg["k"], (cfg["private"] or cfg["M"])
+    R = T * k
+    b = 2
+    return {
+        "route_logits": T * d * b + T * m * 4 + m * d * 4,
+        "route_select": T * m * 4 + T * k * 8 + T * 4,
+        "dispatch_gather": T * d * b + R * d * b + R * 4,
+        "combine": R * d * b + 2 * T * d * b + T * k * 8,
+        "bwd_scale_gather": T * d * b + R * d * b + R * 4,
+        "bwd_dgate": T * d * b + R * d * b + T * k * 8,
+        "unpermute_sum": R * d * b + 2 * T * d * b + T * k * 4,
+    }
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2605_06665_b200 import synth
+    from paper_2605_06665_b200.stack import UniPoolStack
+    import __graft_entry__ as entry
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if rank == 0:
+        entry.build()
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist.barrier()
+    if rank != 0:
+        from paper_2605_06665_b200 import binding
+        binding.lib()
+    dev = torch.device("cuda", local_rank)
+
+    cfg = dict(synth.CONFIGS[args.workload])
+    L, T, d, f, M, k = cfg["L"], cfg["T"], cfg["d"], cfg["f"], cfg["M"], cfg["k"]
+    m = synth.router_width(cfg)
+    inputs = synth.make_inputs(cfg, seed=rank)
+    st = UniPoolStack(L, d, f, M, k, T, cfg["dtype"], cfg["private"], c=1.0, eps=synth.EPS, alpha=synth.ALPHA,
+                      device=dev, deferred_wgrad=args.deferred_wgrad)
+    c_val = st.ctx.calibrate_c(m, k, 100_000, seed=0)          # Alg. 1 on the device
+    st.close()
+    st = UniPoolStack(L, d, f, M, k, T, cfg["dtype"], cfg["private"], c=c_val, eps=synth.EPS, alpha=synth.ALPHA,
+                      device=dev, deferred_wgrad=args.deferred_wgrad)
+    st.load(inputs["pool"], inputs["routers"])
+    tdt = st.tdtype
+    x0_host = torch.from_numpy(inputs["x0"]).to(tdt).pin_memory()
+    up_host = torch.from_numpy(inputs["upstream"]).to(tdt).pin_memory()
+    x0 = x0_host.to(dev)
+    up = up_host.to(dev)
+    xL_host = torch.empty_like(x0_host).pin_memory()
+    loss_host = torch.empty(st.loss.shape, dtype=torch.float32).pin_memory()
+
+    def sync_all():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    def timed(fn, steps):
+        sync_all()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        sync_all()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    def device_step():
+        st.zero_grad()                       # the step's fp32 pool gradient starts at zero
+        st.step(x0, up)
+
+    def e2e_step():
+        st.zero_grad()
+        st.step(x0_host, up_host)            # H2D copies of this step's inputs from pinned memory
+        xL_host.copy_(st.x[L], non_blocking=True)
+        loss_host.copy_(st.loss, non_blocking=True)
+
+    for _ in range(max(args.warmup, 3)):
+        device_step()
+    st.ctx.check_status()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    ms_total = timed(device_step, args.steps)
+    clocks = sampler.stop() if rank == 0 else None
+
+    # per-kernel durations, measured live with CUDA events on the launch stream
+    st.ctx.profile_enable(True)
+    timed(device_step, args.steps)
+    prof = st.ctx.profile_read()
+    st.ctx.profile_enable(False)
+
+    for _ in range(2):
+        e2e_step()
+    ms_e2e = timed(e2e_step, args.steps)
+    st.ctx.check_status()
+
+    ms_step = ms_total / args.steps
+    value = world * T * L / (ms_step * 1e-3)
+    e2e_value = world * T * L / (ms_e2e / args.steps * 1e-3)
+    peaks = _peaks()
+    R = T * k
+    kernels = {}
+    for name, (ms, launches) in prof.items():
+        if launches == 0:
+            continue
+        per_launch_ms = ms / (launches / max(1, {"dispatch_maps": 3}.get(name, 1)))
+        kernels[name] = dict(ms_per_step=ms / args.steps, launches_per_step=launches // args.steps,
+                             ms_per_call=per_launch_ms)
+    abytes = algorithmic_bytes(cfg, st.cap)
+    for name, factor in GEMM_PHASES.items():
+        if name in kernels:
+            flops = factor * R * d * f
+            tf = flops / (kernels[name]["ms_per_call"] * 1e-3) / 1e12
+            kernels[name].update(tflops=tf, frac_of_measured_sustained=tf / peaks["bf16_tflops_sustained"])
+    for name, nbytes in abytes.items():
+        if name in kernels:
+            gbs = nbytes / (kernels[name]["ms_per_call"] * 1e-3) / 1e9
+            kernels[name].update(gbs=gbs, frac_of_measured_hbm=gbs / peaks["hbm_gbs"])
+    gemm_ms = {n: kernels[n]["ms_per_step"] for n in GEMM_PHASES if n in kernels}
+    dominant = max(gemm_ms, key=gemm_ms.get)
+    dom = kernels[dominant]
+    roofline = dict(kernel="grouped_gemm_tc_kernel:" + dominant, bound="tensor", achieved=dom["tflops"],
+                    peak=peaks["bf16_tflops_sustained"], unit="TFLOP/s",
+                    frac=dom["tflops"] / peaks["bf16_tflops_sustained"], peak_source=peaks["source"] + " sustained",
+                    traffic=None)
+    total_gemm_flops = 18 * R * d * f * L
+    gemm_time = sum(gemm_ms.values()) * 1e-3
+    launches = sum(v["launches_per_step"] for v in kernels.values())
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": cfg["dtype"], "data": "synthetic",
+        "config": {"workload": args.workload, "layers": L, "d_model": d, "d_ff": f, "pool_experts": M, "top_k": k,
+                   "tokens_per_gpu": T, "layout": "private" if cfg["private"] else "shared_pool",
+                   "deferred_wgrad": bool(st.deferred_wgrad),
+                   "l2": "working set per step (weights + saved activations, several GB) exceeds the 126 MB L2",
+                   "norm_router_c": c_val},
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": ms_e2e / args.steps,
+                "h2d_bytes_per_step": int(x0_host.numel() * x0_host.element_size() * 2),
+                "d2h_bytes_per_step": int(xL_host.numel() * xL_host.element_size() + loss_host.numel() * 4)},
+        "gpu_launches": launches * args.steps,
+        "roofline": roofline,
+        "stack_tokens_per_s": world * T / (ms_step * 1e-3),
+        "gemm_tflops_all_phases": total_gemm_flops / gemm_time / 1e12,
+        "gemm_frac_of_measured_sustained": total_gemm_flops / gemm_time / 1e12 / peaks["bf16_tflops_sustained"],
+        "kernels": kernels,
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = cpu_baseline(cfg, budget_tokens=args.cpu_tokens)
+    st.close()
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(out))
+
+
+def cpu_baseline(cfg, budget_tokens=2048, repeats=1):
+    """Times the CPU oracle, as it stands, on one MoE layer (forward + backward) over a
+    token sample of the workload; fp32 arithmetic (the arrays it is fed are float32)."""
+    import numpy as np
+    from oracle import unipool_oracle as O
+    from paper_2605_06665_b200 import synth
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        threads = len(os.sched_getaffinity(0))
+    Ts = min(budget_tokens, cfg["T"])
+    inputs = synth.make_inputs(cfg, seed=0, T=Ts, L=1)
+    pool, router = inputs["pool"], inputs["routers"][0]
+    k = cfg["k"]
+    best = None
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        cache = O.layer_forward(inputs["x0"], router, pool, k, np.float32(2.0), np.float32(synth.EPS))
+        _, _, coef = O.pool_aux_loss(cache["counts"][None], cache["S"][None], Ts, k, synth.ALPHA)
+        grad = O.zeros_like_pool(pool)
+        O.layer_backward(cache, router, pool, k, np.float32(2.0), np.float32(synth.EPS), inputs["upstream"],
+                         coef.astype(np.float32), grad)
+        dt = time.perf_counter() - t0
+        best = dt if best is None else min(best, dt)
+    return dict(value=Ts / best, unit=UNIT, cores=int(threads), kind="oracle", seconds=best,
+                sample=f"one MoE layer fwd+bwd (route, Eq. 2, balance-loss term, all gradients) over {Ts} of the "
+                       f"{cfg['T']} tokens, full pool of {cfg['M']} experts, float32 numpy")
+
+
+def run_reference(args):
+    """The reference arm is the oracle (the paper ships no implementation)."""
+    from paper_2605_06665_b200 import synth
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import __graft_entry__ as entry  # noqa: F401  (path set-up)
+    cfg = dict(synth.CONFIGS[args.workload])
+    for _ in range(min(args.warmup, 1)):
+        cpu_baseline(cfg, budget_tokens=min(256, args.cpu_tokens))
+    times = []
+    res = None
+    for _ in range(min(args.steps, 3)):
+        res = cpu_baseline(cfg, budget_tokens=args.cpu_tokens)
+        times.append(res["seconds"])
+    sec = sum(times) / len(times)
+    Ts = min(args.cpu_tokens, cfg["T"])
+    value = Ts / sec
+    out = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT,
+        "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": len(times), "warmup": min(args.warmup, 1),
+        "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": args.workload, "note": "CPU oracle; each step = one MoE layer fwd+bwd over a token sample"},
+        "cpu_baseline": {k: res[k] for k in ("value", "unit", "cores", "kind", "sample")},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(out))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="182m")
+    ap.add_argument("--deferred-wgrad", action="store_true",
+                    help="contract all layers' rows per expert in one pool_wgrad pass at the end of backward")
+    ap.add_argument("--cpu-tokens", type=int, default=16384, help="token sample of the CPU-oracle baseline")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

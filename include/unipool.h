@@ -219,6 +219,22 @@ int unipool_route_bwd(unipool_ctx* ctx, const void* x, int32_t T, const float* W
 int unipool_calibrate_c(unipool_ctx* ctx, int32_t n_experts, int32_t top_k, int32_t n_samples,
                         uint64_t seed, float* c_out, unipool_stream stream);
 
+/* Per-phase device timing (a measurement aid; the paper has no counterpart).
+ * While enabled, every call brackets each of its kernel phases with CUDA events
+ * on the call's stream.  unipool_profile_read synchronises those events, adds the
+ * elapsed milliseconds and kernel-launch counts per phase into ms[] / launches[]
+ * (host arrays of UNIPOOL_N_PHASES entries, overwritten) and forgets them. */
+enum {
+  UNIPOOL_PH_ROUTE_LOGITS = 0, UNIPOOL_PH_ROUTE_SELECT, UNIPOOL_PH_DISPATCH_MAPS,
+  UNIPOOL_PH_DISPATCH_GATHER, UNIPOOL_PH_EXPERT_FWD_GU, UNIPOOL_PH_EXPERT_FWD_DOWN,
+  UNIPOOL_PH_COMBINE, UNIPOOL_PH_POOL_AUX, UNIPOOL_PH_BWD_SCALE_GATHER, UNIPOOL_PH_BWD_DGATE,
+  UNIPOOL_PH_DGRAD_DOWN, UNIPOOL_PH_DGRAD_GU, UNIPOOL_PH_WGRAD_DOWN, UNIPOOL_PH_WGRAD_GU,
+  UNIPOOL_PH_UNPERMUTE_SUM, UNIPOOL_PH_ROUTE_BWD_DZ, UNIPOOL_PH_ROUTE_BWD_DX,
+  UNIPOOL_PH_ROUTE_BWD_DW, UNIPOOL_N_PHASES
+};
+int unipool_profile_enable(unipool_ctx* ctx, int32_t on);
+int unipool_profile_read(unipool_ctx* ctx, double* ms, int64_t* launches);
+
 #ifdef __cplusplus
 }
 #endif

@@ -22,6 +22,13 @@ EXPORTS = (
     "unipool_last_error", "unipool_check_status", "unipool_route", "unipool_dispatch",
     "unipool_expert_fwd", "unipool_combine", "unipool_expert_bwd", "unipool_pool_wgrad",
     "unipool_pool_aux_loss", "unipool_route_bwd", "unipool_calibrate_c",
+    "unipool_profile_enable", "unipool_profile_read",
+)
+
+PHASES = (
+    "route_logits", "route_select", "dispatch_maps", "dispatch_gather", "expert_fwd_gu", "expert_fwd_down",
+    "combine", "pool_aux", "bwd_scale_gather", "bwd_dgate", "dgrad_down", "dgrad_gu", "wgrad_down", "wgrad_gu",
+    "unpermute_sum", "route_bwd_dz", "route_bwd_dx", "route_bwd_dw",
 )
 
 
@@ -85,6 +92,10 @@ def lib():
     L.unipool_route_bwd.argtypes = [vp, vp, i32, vp, f32, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     L.unipool_calibrate_c.restype = ctypes.c_int
     L.unipool_calibrate_c.argtypes = [vp, i32, i32, i32, ctypes.c_uint64, ctypes.POINTER(f32), vp]
+    L.unipool_profile_enable.restype = ctypes.c_int
+    L.unipool_profile_enable.argtypes = [vp, i32]
+    L.unipool_profile_read.restype = ctypes.c_int
+    L.unipool_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i64)]
     _lib = L
     return L
 
@@ -186,6 +197,17 @@ class Context:
         _check(lib().unipool_route_bwd(self.handle, _p(x), T, _p(W_r), sigma, n_experts, _p(znorm),
                                        _p(z_saved), _p(idx), _p(dgate), _p(dscore_coef), _p(dx), _p(dW_r),
                                        _p(dsigma), _stream()))
+
+    def profile_enable(self, on):
+        _check(lib().unipool_profile_enable(self.handle, 1 if on else 0))
+
+    def profile_read(self):
+        """{phase name: (milliseconds, kernel launches)} since the last read."""
+        n = len(PHASES)
+        ms = (ctypes.c_double * n)()
+        launches = (ctypes.c_int64 * n)()
+        _check(lib().unipool_profile_read(self.handle, ms, launches))
+        return {PHASES[i]: (float(ms[i]), int(launches[i])) for i in range(n)}
 
     def calibrate_c(self, n_experts, top_k, n_samples=100_000, seed=0):
         out = ctypes.c_float()

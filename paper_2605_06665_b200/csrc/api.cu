@@ -151,7 +151,31 @@ int unipool_create(unipool_ctx** out, const unipool_config* cfg, void* workspace
 int unipool_destroy(unipool_ctx* ctx) {
   if (!ctx) return UNIPOOL_OK;
   if (ctx->cfg.dtype == UNIPOOL_BF16) tc_module_destroy(ctx);
+  for (const ProfRecord& r : ctx->prof.records) { cudaEventDestroy(r.start); cudaEventDestroy(r.stop); }
+  for (cudaEvent_t e : ctx->prof.free_events) cudaEventDestroy(e);
   delete ctx;
+  return UNIPOOL_OK;
+}
+
+int unipool_profile_enable(unipool_ctx* ctx, int32_t on) {
+  CHECK_CTX(ctx);
+  ctx->prof.enabled = on != 0;
+  return UNIPOOL_OK;
+}
+
+int unipool_profile_read(unipool_ctx* ctx, double* ms, int64_t* launches) {
+  CHECK_CTX(ctx); CHECK_PTR(ms); CHECK_PTR(launches);
+  for (int i = 0; i < UNIPOOL_N_PHASES; ++i) { ms[i] = 0.0; launches[i] = 0; }
+  for (const ProfRecord& r : ctx->prof.records) {
+    UP_CUDA(cudaEventSynchronize(r.stop));
+    float t = 0.f;
+    UP_CUDA(cudaEventElapsedTime(&t, r.start, r.stop));
+    ms[r.phase] += t;
+    launches[r.phase] += r.launches;
+    ctx->prof.free_events.push_back(r.start);
+    ctx->prof.free_events.push_back(r.stop);
+  }
+  ctx->prof.records.clear();
   return UNIPOOL_OK;
 }
 

@@ -35,6 +35,7 @@ pool_aux_kernel(const int32_t* __restrict__ counts, const float* __restrict__ S,
 int aux_launch(unipool_ctx* ctx, const int32_t* counts, const float* S, int L, int M, int T,
                float alpha, const float* fbar_prev, float* loss, float* coef, float* fbar_out,
                cudaStream_t s) {
+  PhaseTimer pt(ctx, UNIPOOL_PH_POOL_AUX, 1, s);
   pool_aux_kernel<<<1, 512, 0, s>>>(counts, S, L, M, T, ctx->cfg.top_k, alpha, fbar_prev, loss, coef,
                                     fbar_out);
   UP_LAUNCH_CHECK();

@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <vector>
+
 #include "unipool.h"
 
 namespace unipool {
@@ -60,7 +62,23 @@ Workspace carve_workspace(const unipool_config& cfg, void* base);
 
 }  // namespace unipool
 
+namespace unipool {
+struct ProfRecord { int phase; int launches; cudaEvent_t start, stop; };
+struct Profiler {
+  bool enabled = false;
+  std::vector<ProfRecord> records;       // events recorded since the last read
+  std::vector<cudaEvent_t> free_events;  // recycled events
+  cudaEvent_t get() {
+    if (!free_events.empty()) { cudaEvent_t e = free_events.back(); free_events.pop_back(); return e; }
+    cudaEvent_t e = nullptr;
+    cudaEventCreate(&e);
+    return e;
+  }
+};
+}  // namespace unipool
+
 struct unipool_ctx {
+  unipool::Profiler prof;
   unipool_config cfg;
   unipool::Workspace ws;
   int device;
@@ -71,6 +89,20 @@ struct unipool_ctx {
 };
 
 namespace unipool {
+
+// Brackets the kernels launched during its lifetime with a pair of events (when profiling is on).
+struct PhaseTimer {
+  unipool_ctx* ctx; cudaStream_t s; cudaEvent_t stop = nullptr;
+  PhaseTimer(unipool_ctx* c, int phase, int launches, cudaStream_t stream) : ctx(c), s(stream) {
+    if (!ctx->prof.enabled) return;
+    cudaEvent_t start = ctx->prof.get();
+    stop = ctx->prof.get();
+    if (!start || !stop) { stop = nullptr; return; }
+    cudaEventRecord(start, s);
+    ctx->prof.records.push_back({phase, launches, start, stop});
+  }
+  ~PhaseTimer() { if (stop) cudaEventRecord(stop, s); }
+};
 
 // ---------------------------------------------------------------- element helpers
 __device__ __forceinline__ float to_f32(float v) { return v; }

@@ -285,12 +285,16 @@ int dispatch_launch(unipool_ctx* ctx, const void* x, int T, const int32_t* idx, 
   }
   const int n_blocks = (T + kDispatchChunkTokens - 1) / kDispatchChunkTokens;
   int32_t* bh = ctx->ws.block_hist;
+  {
+  PhaseTimer pt(ctx, UNIPOOL_PH_DISPATCH_MAPS, 3, s);
   dispatch_hist_kernel<<<n_blocks, 32, M * sizeof(int), s>>>(idx, T, k, M, bh, ctx->ws.status);
   UP_LAUNCH_CHECK();
   dispatch_scan_kernel<<<1, 512, 0, s>>>(bh, n_blocks, M, cap, offsets, token_of, tile_expert);
   UP_LAUNCH_CHECK();
   dispatch_rank_kernel<<<n_blocks, 32, M * sizeof(int), s>>>(idx, T, k, M, bh, row_of, token_of);
   UP_LAUNCH_CHECK();
+  }
+  PhaseTimer pt(ctx, UNIPOOL_PH_DISPATCH_GATHER, 1, s);
   const int row_vecs = (int)((size_t)d * ctx->elem_bytes / 16);
   gather_rows_kernel<<<row_mover_grid(ctx, cap), 256, 0, s>>>(
       static_cast<const uint4*>(x), token_of, offsets + M, static_cast<uint4*>(Xp), row_vecs, cap);
@@ -298,9 +302,10 @@ int dispatch_launch(unipool_ctx* ctx, const void* x, int T, const int32_t* idx, 
   return UNIPOOL_OK;
 }
 
-int combine_launch(unipool_ctx* ctx, const void* Yp, const int32_t* row_of, const float* gate, int T,
-                   const void* residual, void* y, cudaStream_t s) {
+static int combine_phase(unipool_ctx* ctx, int phase, const void* Yp, const int32_t* row_of,
+                         const float* gate, int T, const void* residual, void* y, cudaStream_t s) {
   if (T == 0) return UNIPOOL_OK;
+  PhaseTimer pt(ctx, phase, 1, s);
   const int k = ctx->cfg.top_k;
   const int row_vecs = (int)((size_t)ctx->cfg.d_model * ctx->elem_bytes / 16);
   const int grid = row_mover_grid(ctx, T);
@@ -314,6 +319,11 @@ int combine_launch(unipool_ctx* ctx, const void* Yp, const int32_t* row_of, cons
   return UNIPOOL_OK;
 }
 
+int combine_launch(unipool_ctx* ctx, const void* Yp, const int32_t* row_of, const float* gate, int T,
+                   const void* residual, void* y, cudaStream_t s) {
+  return combine_phase(ctx, UNIPOOL_PH_COMBINE, Yp, row_of, gate, T, residual, y, s);
+}
+
 int combine_bwd_launch(unipool_ctx* ctx, const void* dy, int T, const int32_t* row_of,
                        const float* gate, const int32_t* token_of, const int32_t* offsets, int M,
                        const void* Yp, void* dYp, float* dgate, cudaStream_t s) {
@@ -321,19 +331,24 @@ int combine_bwd_launch(unipool_ctx* ctx, const void* dy, int T, const int32_t* r
   const int k = ctx->cfg.top_k;
   const int row_vecs = (int)((size_t)ctx->cfg.d_model * ctx->elem_bytes / 16);
   const int g1 = row_mover_grid(ctx, ctx->row_capacity), g2 = row_mover_grid(ctx, T);
-  if (ctx->cfg.dtype == UNIPOOL_BF16) {
-    scale_gather_kernel<__nv_bfloat16><<<g1, 256, 0, s>>>(static_cast<const uint4*>(dy), token_of, row_of,
-        gate, offsets + M, static_cast<uint4*>(dYp), k, row_vecs);
+  const bool bf16 = ctx->cfg.dtype == UNIPOOL_BF16;
+  {
+    PhaseTimer pt(ctx, UNIPOOL_PH_BWD_SCALE_GATHER, 1, s);
+    if (bf16)
+      scale_gather_kernel<__nv_bfloat16><<<g1, 256, 0, s>>>(static_cast<const uint4*>(dy), token_of, row_of,
+          gate, offsets + M, static_cast<uint4*>(dYp), k, row_vecs);
+    else
+      scale_gather_kernel<float><<<g1, 256, 0, s>>>(static_cast<const uint4*>(dy), token_of, row_of, gate,
+          offsets + M, static_cast<uint4*>(dYp), k, row_vecs);
     UP_LAUNCH_CHECK();
+  }
+  PhaseTimer pt(ctx, UNIPOOL_PH_BWD_DGATE, 1, s);
+  if (bf16)
     dgate_kernel<__nv_bfloat16><<<g2, 256, 0, s>>>(static_cast<const uint4*>(dy), static_cast<const uint4*>(Yp),
         row_of, dgate, T, k, row_vecs);
-  } else {
-    scale_gather_kernel<float><<<g1, 256, 0, s>>>(static_cast<const uint4*>(dy), token_of, row_of, gate,
-        offsets + M, static_cast<uint4*>(dYp), k, row_vecs);
-    UP_LAUNCH_CHECK();
+  else
     dgate_kernel<float><<<g2, 256, 0, s>>>(static_cast<const uint4*>(dy), static_cast<const uint4*>(Yp),
         row_of, dgate, T, k, row_vecs);
-  }
   UP_LAUNCH_CHECK();
   return UNIPOOL_OK;
 }
@@ -341,7 +356,7 @@ int combine_bwd_launch(unipool_ctx* ctx, const void* dy, int T, const int32_t* r
 int unpermute_sum_launch(unipool_ctx* ctx, const void* dXp, const int32_t* row_of, int T,
                          const void* residual, void* dx, cudaStream_t s) {
   // dx_t = residual_t + sum_j dXp[row_of[t,j]]: the combine kernel with unit weights
-  return combine_launch(ctx, dXp, row_of, nullptr, T, residual, dx, s);
+  return combine_phase(ctx, UNIPOOL_PH_UNPERMUTE_SUM, dXp, row_of, nullptr, T, residual, dx, s);
 }
 
 }  // namespace unipool

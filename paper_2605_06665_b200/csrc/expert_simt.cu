@@ -108,11 +108,15 @@ static int fwd_impl(unipool_ctx* ctx, const ExpertFwdArgs& a, cudaStream_t s) {
   TE* A = static_cast<TE*>(a.A);
   TE* Yp = static_cast<TE*>(a.Yp);
   // GU = Xp W_gu[e]^T : B(k, n) = W_gu[e][n, k]
+  {
+  PhaseTimer pt(ctx, UNIPOOL_PH_EXPERT_FWD_GU, 2, s);
   grouped_rows_gemm_kernel<TE><<<dim3(2 * f / kSimtTile, gy), kSimtThreads, 0, s>>>(
       Xp, d, Wgu, (int64_t)2 * f * d, 1, d, a.tile_expert, a.expert_base, GU, 2 * f, 2 * f, d, n_row_tiles);
   UP_LAUNCH_CHECK();
   swiglu_kernel<TE><<<ctx->sm_count * 8, 256, 0, s>>>(GU, A, a.offsets + a.n_experts, f);
   UP_LAUNCH_CHECK();
+  }
+  PhaseTimer pt(ctx, UNIPOOL_PH_EXPERT_FWD_DOWN, 1, s);
   // Yp = A W_down[e]^T : B(k, n) = W_down[e][n, k]
   grouped_rows_gemm_kernel<TE><<<dim3(d / kSimtTile, gy), kSimtThreads, 0, s>>>(
       A, f, Wd, (int64_t)d * f, 1, f, a.tile_expert, a.expert_base, Yp, d, d, f, n_row_tiles);
@@ -124,10 +128,14 @@ template <typename TE>
 static int wgrad_impl(unipool_ctx* ctx, const PoolWgradArgs& a, cudaStream_t s) {
   const int d = ctx->cfg.d_model, f = ctx->cfg.d_ff;
   // dW_down[e][d, f] += dYp_e^T A_e
+  {
+  PhaseTimer pt(ctx, UNIPOOL_PH_WGRAD_DOWN, 1, s);
   grouped_k_gemm_kernel<TE><<<dim3(d / kSimtTile, f / kSimtTile, a.n_experts), kSimtThreads, 0, s>>>(
       static_cast<const TE*>(a.dYp), d, static_cast<const TE*>(a.A), f, a.offsets, a.n_experts,
       a.expert_base, a.n_layers, a.layer_stride_rows, a.dW_down, (int64_t)d * f, d, f);
   UP_LAUNCH_CHECK();
+  }
+  PhaseTimer pt(ctx, UNIPOOL_PH_WGRAD_GU, 1, s);
   // dW_gu[e][2f, d] += dGU_e^T Xp_e
   grouped_k_gemm_kernel<TE><<<dim3(2 * f / kSimtTile, d / kSimtTile, a.n_experts), kSimtThreads, 0, s>>>(
       static_cast<const TE*>(a.dGU), 2 * f, static_cast<const TE*>(a.Xp), d, a.offsets, a.n_experts,
@@ -144,6 +152,8 @@ static int bwd_impl(unipool_ctx* ctx, const ExpertBwdArgs& a, cudaStream_t s) {
   const TE* dYp = static_cast<const TE*>(a.dYp);
   TE* dGU = static_cast<TE*>(a.dGU);
   // dA = dYp W_down[e] : B(k, n) = W_down[e][k, n]; lands in the U half of dGU
+  {
+  PhaseTimer pt(ctx, UNIPOOL_PH_DGRAD_DOWN, 2, s);
   grouped_rows_gemm_kernel<TE><<<dim3(f / kSimtTile, gy), kSimtThreads, 0, s>>>(
       dYp, d, static_cast<const TE*>(a.W_down), (int64_t)d * f, f, 1, a.tile_expert, a.expert_base,
       dGU + f, 2 * f, f, d, n_row_tiles);
@@ -151,11 +161,15 @@ static int bwd_impl(unipool_ctx* ctx, const ExpertBwdArgs& a, cudaStream_t s) {
   swiglu_bwd_kernel<TE><<<ctx->sm_count * 8, 256, 0, s>>>(static_cast<const TE*>(a.GU), dGU,
                                                           a.offsets + a.n_experts, f);
   UP_LAUNCH_CHECK();
+  }
   // dXp = dGU W_gu[e] : B(k, n) = W_gu[e][k, n]
+  {
+  PhaseTimer pt(ctx, UNIPOOL_PH_DGRAD_GU, 1, s);
   grouped_rows_gemm_kernel<TE><<<dim3(d / kSimtTile, gy), kSimtThreads, 0, s>>>(
       dGU, 2 * f, static_cast<const TE*>(a.W_gu), (int64_t)2 * f * d, d, 1, a.tile_expert,
       a.expert_base, static_cast<TE*>(a.dXp), d, d, 2 * f, n_row_tiles);
   UP_LAUNCH_CHECK();
+  }
   if (a.wgrad) {
     PoolWgradArgs w{1, 0, a.offsets, a.Xp, a.A, a.dYp, a.dGU, a.expert_base, a.n_experts, a.dW_gu, a.dW_down};
     return wgrad_impl<TE>(ctx, w, s);

@@ -419,7 +419,9 @@ int map_2d(const unipool_ctx* ctx, CUtensorMap* out, const void* base, uint64_t 
 }
 
 template <int MODE, int BN>
-int launch(unipool_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmParams& p, cudaStream_t s) {
+int launch(unipool_ctx* ctx, int phase, const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmParams& p,
+           cudaStream_t s) {
+  PhaseTimer pt(ctx, phase, 1, s);
   auto kern = grouped_gemm_tc_kernel<MODE, BN>;
   constexpr int smem = SmemLayout<BN>::kTotal;
   UP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
@@ -444,12 +446,12 @@ int wgrad_pair(unipool_ctx* ctx, const PoolWgradArgs& a, cudaStream_t s) {
   if ((rc = map_2d(ctx, &tmP, a.dYp, d, rows, 64, 64)) != UNIPOOL_OK) return rc;
   if ((rc = map_2d(ctx, &tmQ, a.A, f, rows, 64, 64)) != UNIPOOL_OK) return rc;
   p.Mdim = d; p.Ndim = f; p.dW = a.dW_down;
-  if ((rc = launch<kWgrad, 128>(ctx, tmP, tmQ, p, s)) != UNIPOOL_OK) return rc;
+  if ((rc = launch<kWgrad, 128>(ctx, UNIPOOL_PH_WGRAD_DOWN, tmP, tmQ, p, s)) != UNIPOOL_OK) return rc;
   // dW_gu[e] [2f, d] += dGU_e^T Xp_e
   if ((rc = map_2d(ctx, &tmP, a.dGU, 2 * f, rows, 64, 64)) != UNIPOOL_OK) return rc;
   if ((rc = map_2d(ctx, &tmQ, a.Xp, d, rows, 64, 64)) != UNIPOOL_OK) return rc;
   p.Mdim = 2 * f; p.Ndim = d; p.dW = a.dW_gu;
-  return launch<kWgrad, 128>(ctx, tmP, tmQ, p, s);
+  return launch<kWgrad, 128>(ctx, UNIPOOL_PH_WGRAD_GU, tmP, tmQ, p, s);
 }
 
 }  // namespace
@@ -494,14 +496,14 @@ int expert_fwd_tc(unipool_ctx* ctx, const ExpertFwdArgs& a, cudaStream_t s) {
   p.Ndim = f; p.Kdim = d;
   p.out0 = static_cast<__nv_bfloat16*>(a.GU);
   p.out1 = static_cast<__nv_bfloat16*>(a.A);
-  if ((rc = launch<kFwd1, 128>(ctx, tmA, tmB, p, s)) != UNIPOOL_OK) return rc;
+  if ((rc = launch<kFwd1, 128>(ctx, UNIPOOL_PH_EXPERT_FWD_GU, tmA, tmB, p, s)) != UNIPOOL_OK) return rc;
   // Yp = A W_down^T
   if ((rc = map_2d(ctx, &tmA, a.A, f, cap, 64, 128)) != UNIPOOL_OK) return rc;
   if ((rc = map_2d(ctx, &tmB, a.W_down, f, (uint64_t)M * d, 64, 128)) != UNIPOOL_OK) return rc;
   p.Ndim = d; p.Kdim = f;
   p.out0 = static_cast<__nv_bfloat16*>(a.Yp);
   p.out1 = nullptr;
-  return launch<kFwd2, 128>(ctx, tmA, tmB, p, s);
+  return launch<kFwd2, 128>(ctx, UNIPOOL_PH_EXPERT_FWD_DOWN, tmA, tmB, p, s);
 }
 
 int expert_bwd_tc(unipool_ctx* ctx, const ExpertBwdArgs& a, cudaStream_t s) {
@@ -522,13 +524,13 @@ int expert_bwd_tc(unipool_ctx* ctx, const ExpertBwdArgs& a, cudaStream_t s) {
   p.Ndim = f; p.Kdim = d;
   p.GU = static_cast<const __nv_bfloat16*>(a.GU);
   p.out0 = static_cast<__nv_bfloat16*>(a.dGU);
-  if ((rc = launch<kDgrad1, 128>(ctx, tmA, tmB, p, s)) != UNIPOOL_OK) return rc;
+  if ((rc = launch<kDgrad1, 128>(ctx, UNIPOOL_PH_DGRAD_DOWN, tmA, tmB, p, s)) != UNIPOOL_OK) return rc;
   // dXp = dGU [W_gate; W_up]
   if ((rc = map_2d(ctx, &tmA, a.dGU, 2 * f, cap, 64, 128)) != UNIPOOL_OK) return rc;
   if ((rc = map_2d(ctx, &tmB, a.W_gu, d, (uint64_t)M * 2 * f, 64, 64)) != UNIPOOL_OK) return rc;
   p.Ndim = d; p.Kdim = 2 * f;
   p.out0 = static_cast<__nv_bfloat16*>(a.dXp);
-  if ((rc = launch<kDgrad2, 128>(ctx, tmA, tmB, p, s)) != UNIPOOL_OK) return rc;
+  if ((rc = launch<kDgrad2, 128>(ctx, UNIPOOL_PH_DGRAD_GU, tmA, tmB, p, s)) != UNIPOOL_OK) return rc;
   if (a.wgrad) {
     PoolWgradArgs w{1, 0, a.offsets, a.Xp, a.A, a.dYp, a.dGU, a.expert_base, a.n_experts, a.dW_gu, a.dW_down};
     return wgrad_pair(ctx, w, s);

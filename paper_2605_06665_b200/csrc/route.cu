@@ -136,6 +136,8 @@ int route_launch(unipool_ctx* ctx, const void* x, int T, const float* W_r, float
     return UNIPOOL_OK;
   }
   dim3 g1((T + kSimtTile - 1) / kSimtTile, (M + kSimtTile - 1) / kSimtTile);
+  {
+  PhaseTimer pt(ctx, UNIPOOL_PH_ROUTE_LOGITS, 1, s);
   if (ctx->cfg.dtype == UNIPOOL_BF16)
     router_logits_kernel<__nv_bfloat16><<<g1, kSimtThreads, 0, s>>>(
         static_cast<const __nv_bfloat16*>(x), W_r, bias, z_saved, T, M, d);
@@ -143,6 +145,8 @@ int route_launch(unipool_ctx* ctx, const void* x, int T, const float* W_r, float
     router_logits_kernel<float><<<g1, kSimtThreads, 0, s>>>(static_cast<const float*>(x), W_r, bias,
                                                             z_saved, T, M, d);
   UP_LAUNCH_CHECK();
+  }
+  PhaseTimer pt(ctx, UNIPOOL_PH_ROUTE_SELECT, 1, s);
   const int per_block = kRouteWarps * kRouteTokensPerWarp;
   const int blocks = (T + per_block - 1) / per_block;
   const size_t smem = (size_t)(2 * kRouteWarps * M) * sizeof(float) + (size_t)M * sizeof(int);
@@ -278,22 +282,30 @@ int route_bwd_launch(unipool_ctx* ctx, const void* x, int T, const float* W_r, f
   if (T == 0) return UNIPOOL_OK;
   const int d = ctx->cfg.d_model, k = ctx->cfg.top_k;
   float* dz = ctx->ws.dz;
+  {
+  PhaseTimer pt(ctx, UNIPOOL_PH_ROUTE_BWD_DZ, 1, s);
   router_dz_kernel<<<(T + 7) / 8, 256, 0, s>>>(z_saved, znorm, idx, dgate, coef, T, M, k, sigma,
                                                ctx->cfg.c, ctx->cfg.eps, dz, dsigma,
                                                ctx->ws.dsigma_acc, ctx->ws.tickets + 1);
   UP_LAUNCH_CHECK();
+  }
   dim3 g2((T + kSimtTile - 1) / kSimtTile, d / kSimtTile);
   const int k_len = 1024;
   dim3 g3((M + kSimtTile - 1) / kSimtTile, d / kSimtTile, (T + k_len - 1) / k_len);
-  if (ctx->cfg.dtype == UNIPOOL_BF16) {
-    router_dx_kernel<__nv_bfloat16><<<g2, kSimtThreads, 0, s>>>(dz, W_r, static_cast<__nv_bfloat16*>(dx), T, M, d);
+  const bool bf16 = ctx->cfg.dtype == UNIPOOL_BF16;
+  {
+    PhaseTimer pt(ctx, UNIPOOL_PH_ROUTE_BWD_DX, 1, s);
+    if (bf16)
+      router_dx_kernel<__nv_bfloat16><<<g2, kSimtThreads, 0, s>>>(dz, W_r, static_cast<__nv_bfloat16*>(dx), T, M, d);
+    else
+      router_dx_kernel<float><<<g2, kSimtThreads, 0, s>>>(dz, W_r, static_cast<float*>(dx), T, M, d);
     UP_LAUNCH_CHECK();
-    router_dw_kernel<__nv_bfloat16><<<g3, kSimtThreads, 0, s>>>(dz, static_cast<const __nv_bfloat16*>(x), dW_r, T, M, d, k_len);
-  } else {
-    router_dx_kernel<float><<<g2, kSimtThreads, 0, s>>>(dz, W_r, static_cast<float*>(dx), T, M, d);
-    UP_LAUNCH_CHECK();
-    router_dw_kernel<float><<<g3, kSimtThreads, 0, s>>>(dz, static_cast<const float*>(x), dW_r, T, M, d, k_len);
   }
+  PhaseTimer pt(ctx, UNIPOOL_PH_ROUTE_BWD_DW, 1, s);
+  if (bf16)
+    router_dw_kernel<__nv_bfloat16><<<g3, kSimtThreads, 0, s>>>(dz, static_cast<const __nv_bfloat16*>(x), dW_r, T, M, d, k_len);
+  else
+    router_dw_kernel<float><<<g3, kSimtThreads, 0, s>>>(dz, static_cast<const float*>(x), dW_r, T, M, d, k_len);
   UP_LAUNCH_CHECK();
   return UNIPOOL_OK;
 }
