@@ -176,12 +176,12 @@ def run_ours(args):
         return ms
 
     def device_step():
-        st.zero_grad()                       # the step's fp32 pool gradient starts at zero
-        st.step(x0, up)
+        # the step's first weight-gradient contribution overwrites the fp32 pool gradient, so it
+        # needs no zeroing; the (small) router gradients are zeroed inside the step
+        st.step(x0, up, accumulate=False)
 
     def e2e_step():
-        st.zero_grad()
-        st.step(x0_host, up_host)            # H2D copies of this step's inputs from pinned memory
+        st.step(x0_host, up_host, accumulate=False)   # H2D copies of this step's inputs from pinned memory
         xL_host.copy_(st.x[L], non_blocking=True)
         loss_host.copy_(st.loss, non_blocking=True)
 
@@ -335,8 +335,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="182m")
-    ap.add_argument("--deferred-wgrad", action="store_true",
-                    help="contract all layers' rows per expert in one pool_wgrad pass at the end of backward")
+    ap.add_argument("--per-layer-wgrad", dest="deferred_wgrad", action="store_false",
+                    help="accumulate each layer's weight gradient into the pool gradient during that layer's "
+                         "backward instead of contracting all layers' rows per expert in one pass at the end")
     ap.add_argument("--cpu-tokens", type=int, default=16384, help="token sample of the CPU-oracle baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

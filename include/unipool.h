@@ -59,6 +59,9 @@ extern "C" {
 /* expert_bwd flags */
 #define UNIPOOL_BWD_DEFAULT     0
 #define UNIPOOL_BWD_SKIP_WGRAD  1     /* leave dW to a later unipool_pool_wgrad     */
+#define UNIPOOL_WGRAD_OVERWRITE 2     /* dW of the experts in the view is written,  */
+                                      /* not added to: the first contribution of a  */
+                                      /* step needs no zeroed buffer and no read    */
 
 typedef struct unipool_ctx unipool_ctx;
 typedef void* unipool_stream;         /* a cudaStream_t                            */
@@ -164,7 +167,9 @@ int unipool_combine(unipool_ctx* ctx, const void* Yp, const int32_t* row_of, con
  *      they are the operands a deferred unipool_pool_wgrad needs).
  * out: dx [T,d] (ctx dtype, overwritten); dgate [T,k] float (overwritten);
  *      dW_gu [M,2f,d] float +=; dW_down [M,d,f] float += (skipped when flags has
- *      UNIPOOL_BWD_SKIP_WGRAD; the pointers may then be NULL). */
+ *      UNIPOOL_BWD_SKIP_WGRAD, the pointers may then be NULL; with
+ *      UNIPOOL_WGRAD_OVERWRITE the slices of experts expert_base ..
+ *      expert_base+n_experts-1 are overwritten, zeros for an expert without rows). */
 int unipool_expert_bwd(unipool_ctx* ctx, const void* dy, int32_t T, const int32_t* row_of,
                        const float* gate, const int32_t* token_of, const int32_t* offsets,
                        const int32_t* tile_expert, const void* Xp, const void* GU, const void* A,
@@ -179,11 +184,11 @@ int unipool_expert_bwd(unipool_ctx* ctx, const void* dy, int32_t T, const int32_
  * the per-layer accumulation of unipool_expert_bwd up to summation order).
  * The per-layer operands are slices of stacked buffers: layer l's Xp is
  * Xp + l*layer_stride_rows*d elements, likewise A, dYp, dGU; offsets is
- * [n_layers, n_experts+1]. */
+ * [n_layers, n_experts+1].  flags: 0 (dW +=) or UNIPOOL_WGRAD_OVERWRITE (dW =). */
 int unipool_pool_wgrad(unipool_ctx* ctx, int32_t n_layers, int64_t layer_stride_rows,
                        const int32_t* offsets, const void* Xp, const void* A, const void* dYp,
                        const void* dGU, int32_t expert_base, int32_t n_experts, float* dW_gu,
-                       float* dW_down, unipool_stream stream);
+                       float* dW_down, int32_t flags, unipool_stream stream);
 
 /* Pool-level balance loss (Eqs. 4-5; Eq. 3 when L = 1):
  *   f^(l) = counts^(l) / (T k),  P^(l) = score_sum^(l) / T,  fbar, Pbar = means over l,

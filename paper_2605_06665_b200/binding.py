@@ -16,6 +16,7 @@ LIB_PATH = os.path.join(_HERE, "libunipool.so")
 FP32, BF16 = 0, 1
 ROW_ALIGN = 128
 BWD_SKIP_WGRAD = 1
+WGRAD_OVERWRITE = 2
 
 EXPORTS = (
     "unipool_row_capacity", "unipool_workspace_bytes", "unipool_create", "unipool_destroy",
@@ -85,7 +86,7 @@ def lib():
     L.unipool_expert_bwd.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32,
                                      vp, vp, vp, vp, vp, vp, vp, i32, vp]
     L.unipool_pool_wgrad.restype = ctypes.c_int
-    L.unipool_pool_wgrad.argtypes = [vp, i32, i64, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp]
+    L.unipool_pool_wgrad.argtypes = [vp, i32, i64, vp, vp, vp, vp, vp, i32, i32, vp, vp, i32, vp]
     L.unipool_pool_aux_loss.restype = ctypes.c_int
     L.unipool_pool_aux_loss.argtypes = [vp, vp, vp, i32, i32, i32, f32, vp, vp, vp, vp, vp]
     L.unipool_route_bwd.restype = ctypes.c_int
@@ -184,10 +185,10 @@ class Context:
                                         flags, _stream()))
 
     def pool_wgrad(self, n_layers, layer_stride_rows, offsets, Xp, A, dYp, dGU, expert_base, n_experts,
-                   dW_gu, dW_down):
+                   dW_gu, dW_down, flags=0):
         _check(lib().unipool_pool_wgrad(self.handle, n_layers, layer_stride_rows, _p(offsets), _p(Xp), _p(A),
                                         _p(dYp), _p(dGU), expert_base, n_experts, _p(dW_gu), _p(dW_down),
-                                        _stream()))
+                                        flags, _stream()))
 
     def pool_aux_loss(self, counts, score_sum, L, n_experts, T, alpha, fbar_prev, loss, dscore_coef, fbar_out):
         _check(lib().unipool_pool_aux_loss(self.handle, _p(counts), _p(score_sum), L, n_experts, T, alpha,

@@ -247,14 +247,15 @@ int unipool_expert_bwd(unipool_ctx* ctx, const void* dy, int32_t T, const int32_
   CHECK_PTR(dy); CHECK_PTR(row_of); CHECK_PTR(gate); CHECK_PTR(token_of); CHECK_PTR(offsets);
   CHECK_PTR(tile_expert); CHECK_PTR(Xp); CHECK_PTR(GU); CHECK_PTR(A); CHECK_PTR(Yp);
   CHECK_PTR(W_gu); CHECK_PTR(W_down); CHECK_PTR(dYp); CHECK_PTR(dGU); CHECK_PTR(dx); CHECK_PTR(dgate);
-  UP_REQUIRE((flags & ~UNIPOOL_BWD_SKIP_WGRAD) == 0, UNIPOOL_ERR_INVALID_ARG, "unknown flags 0x%x", flags);
+  UP_REQUIRE((flags & ~(UNIPOOL_BWD_SKIP_WGRAD | UNIPOOL_WGRAD_OVERWRITE)) == 0, UNIPOOL_ERR_INVALID_ARG,
+             "unknown flags 0x%x", flags);
   const bool wgrad = !(flags & UNIPOOL_BWD_SKIP_WGRAD);
   if (wgrad) { CHECK_PTR(dW_gu); CHECK_PTR(dW_down); }
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   int rc = combine_bwd_launch(ctx, dy, T, row_of, gate, token_of, offsets, n_experts, Yp, dYp, dgate, s);
   if (rc != UNIPOOL_OK) return rc;
   ExpertBwdArgs a{offsets, tile_expert, Xp, GU, A, W_gu, W_down, expert_base, n_experts,
-                  dYp, dGU, ctx->ws.dXp, dW_gu, dW_down, wgrad};
+                  dYp, dGU, ctx->ws.dXp, dW_gu, dW_down, wgrad, (flags & UNIPOOL_WGRAD_OVERWRITE) != 0};
   rc = use_tensor_cores(ctx) ? expert_bwd_tc(ctx, a, s) : expert_bwd_simt(ctx, a, s);
   if (rc != UNIPOOL_OK) return rc;
   return unpermute_sum_launch(ctx, ctx->ws.dXp, row_of, T, dx_residual, dx, s);
@@ -263,15 +264,16 @@ int unipool_expert_bwd(unipool_ctx* ctx, const void* dy, int32_t T, const int32_
 int unipool_pool_wgrad(unipool_ctx* ctx, int32_t n_layers, int64_t layer_stride_rows,
                        const int32_t* offsets, const void* Xp, const void* A, const void* dYp,
                        const void* dGU, int32_t expert_base, int32_t n_experts, float* dW_gu,
-                       float* dW_down, unipool_stream stream) {
+                       float* dW_down, int32_t flags, unipool_stream stream) {
   CHECK_CTX(ctx); CHECK_VIEW(ctx, expert_base, n_experts);
   UP_REQUIRE(n_layers >= 1, UNIPOOL_ERR_INVALID_ARG, "n_layers must be >= 1");
   UP_REQUIRE(layer_stride_rows >= 0 && layer_stride_rows % UNIPOOL_ROW_ALIGN == 0,
              UNIPOOL_ERR_INVALID_ARG, "layer_stride_rows must be a multiple of %d", UNIPOOL_ROW_ALIGN);
   CHECK_PTR(offsets); CHECK_PTR(Xp); CHECK_PTR(A); CHECK_PTR(dYp); CHECK_PTR(dGU);
   CHECK_PTR(dW_gu); CHECK_PTR(dW_down);
+  UP_REQUIRE((flags & ~UNIPOOL_WGRAD_OVERWRITE) == 0, UNIPOOL_ERR_INVALID_ARG, "unknown flags 0x%x", flags);
   PoolWgradArgs a{n_layers, layer_stride_rows, offsets, Xp, A, dYp, dGU, expert_base, n_experts,
-                  dW_gu, dW_down};
+                  dW_gu, dW_down, (flags & UNIPOOL_WGRAD_OVERWRITE) != 0};
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   return use_tensor_cores(ctx) ? pool_wgrad_tc(ctx, a, s) : pool_wgrad_simt(ctx, a, s);
 }

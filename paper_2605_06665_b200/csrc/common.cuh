@@ -157,12 +157,12 @@ struct ExpertBwdArgs {
   const int32_t* offsets; const int32_t* tile_expert;
   const void* Xp; const void* GU; const void* A; const void* W_gu; const void* W_down;
   int expert_base; int n_experts;
-  const void* dYp; void* dGU; void* dXp; float* dW_gu; float* dW_down; bool wgrad;
+  const void* dYp; void* dGU; void* dXp; float* dW_gu; float* dW_down; bool wgrad; bool overwrite;
 };
 struct PoolWgradArgs {
   int n_layers; int64_t layer_stride_rows; const int32_t* offsets;
   const void* Xp; const void* A; const void* dYp; const void* dGU;
-  int expert_base; int n_experts; float* dW_gu; float* dW_down;
+  int expert_base; int n_experts; float* dW_gu; float* dW_down; bool overwrite;
 };
 int expert_fwd_simt(unipool_ctx*, const ExpertFwdArgs&, cudaStream_t);
 int expert_bwd_simt(unipool_ctx*, const ExpertBwdArgs&, cudaStream_t);

@@ -40,7 +40,7 @@ __global__ void __launch_bounds__(kSimtThreads)
 grouped_k_gemm_kernel(const TE* __restrict__ P, int64_t ldp, const TE* __restrict__ Q, int64_t ldq,
                       const int32_t* __restrict__ offsets, int n_experts, int expert_base,
                       int n_layers, int64_t layer_stride_rows, float* __restrict__ dW,
-                      int64_t w_expert_stride, int Mdim, int Ndim) {
+                      int64_t w_expert_stride, int Mdim, int Ndim, bool overwrite) {
   const int m0 = blockIdx.x * kSimtTile, n0 = blockIdx.y * kSimtTile;
   const int e = blockIdx.z;
   float acc[4][4] = {};
@@ -62,7 +62,7 @@ grouped_k_gemm_kernel(const TE* __restrict__ P, int64_t ldp, const TE* __restric
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       int n = n0 + tx * 4 + j;
-      if (n < Ndim) out[(int64_t)m * Ndim + n] += acc[i][j];
+      if (n < Ndim) out[(int64_t)m * Ndim + n] = overwrite ? acc[i][j] : out[(int64_t)m * Ndim + n] + acc[i][j];
     }
   }
 }
@@ -132,14 +132,14 @@ static int wgrad_impl(unipool_ctx* ctx, const PoolWgradArgs& a, cudaStream_t s) 
   PhaseTimer pt(ctx, UNIPOOL_PH_WGRAD_DOWN, 1, s);
   grouped_k_gemm_kernel<TE><<<dim3(d / kSimtTile, f / kSimtTile, a.n_experts), kSimtThreads, 0, s>>>(
       static_cast<const TE*>(a.dYp), d, static_cast<const TE*>(a.A), f, a.offsets, a.n_experts,
-      a.expert_base, a.n_layers, a.layer_stride_rows, a.dW_down, (int64_t)d * f, d, f);
+      a.expert_base, a.n_layers, a.layer_stride_rows, a.dW_down, (int64_t)d * f, d, f, a.overwrite);
   UP_LAUNCH_CHECK();
   }
   PhaseTimer pt(ctx, UNIPOOL_PH_WGRAD_GU, 1, s);
   // dW_gu[e][2f, d] += dGU_e^T Xp_e
   grouped_k_gemm_kernel<TE><<<dim3(2 * f / kSimtTile, d / kSimtTile, a.n_experts), kSimtThreads, 0, s>>>(
       static_cast<const TE*>(a.dGU), 2 * f, static_cast<const TE*>(a.Xp), d, a.offsets, a.n_experts,
-      a.expert_base, a.n_layers, a.layer_stride_rows, a.dW_gu, (int64_t)2 * f * d, 2 * f, d);
+      a.expert_base, a.n_layers, a.layer_stride_rows, a.dW_gu, (int64_t)2 * f * d, 2 * f, d, a.overwrite);
   UP_LAUNCH_CHECK();
   return UNIPOOL_OK;
 }
@@ -171,7 +171,8 @@ static int bwd_impl(unipool_ctx* ctx, const ExpertBwdArgs& a, cudaStream_t s) {
   UP_LAUNCH_CHECK();
   }
   if (a.wgrad) {
-    PoolWgradArgs w{1, 0, a.offsets, a.Xp, a.A, a.dYp, a.dGU, a.expert_base, a.n_experts, a.dW_gu, a.dW_down};
+    PoolWgradArgs w{1, 0, a.offsets, a.Xp, a.A, a.dYp, a.dGU, a.expert_base, a.n_experts, a.dW_gu, a.dW_down,
+                    a.overwrite};
     return wgrad_impl<TE>(ctx, w, s);
   }
   return UNIPOOL_OK;

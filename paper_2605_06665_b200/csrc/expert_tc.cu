@@ -20,17 +20,26 @@ namespace unipool {
 namespace {
 
 constexpr int BM = 128;          // rows of an output tile (TMEM lanes)
+constexpr int BN = 256;          // columns of an output tile (one tcgen05.mma of N = 256)
 constexpr int BK = 64;           // k-block: 64 bf16 = one 128-byte swizzle row
 constexpr int kThreads = 192;
+constexpr int kEpiWarps = 4;
 constexpr uint32_t kABytes = BM * BK * 2;
+constexpr uint32_t kBBytes = BN * BK * 2;
+constexpr uint32_t kStageBytes = kABytes + kBBytes;
 constexpr uint32_t kMnBlockBytes = 64 * BK * 2;   // one 64(MN) x 64(K) box
+constexpr uint32_t kBarOffset = 229376;           // operand stages + epilogue staging fill this much
+constexpr uint32_t kSmemTotal = kBarOffset + 512 + 1024;   // + barriers + alignment slack
+constexpr int kChunk = 32;       // output columns one epilogue step moves (a 32 x 32 box per warp)
+constexpr uint32_t kBf16ChunkBytes = 32 * kChunk * 2;      // 2 KiB, 64-byte rows, 64-byte swizzle
+constexpr uint32_t kF32ChunkBytes = 32 * kChunk * 4;       // 4 KiB, 128-byte rows, 128-byte swizzle
 
 enum Mode : int {
   kFwd1 = 0,    // GU = Xp W_gu^T, A = silu(G)*U        A K-major, B K-major (3-D map), row tiles
   kFwd2 = 1,    // Yp = A W_down^T                      A K-major, B K-major,           row tiles
   kDgrad1 = 2,  // dGU = swiglu'(dYp W_down, GU)        A K-major, B MN-major,          row tiles
   kDgrad2 = 3,  // dXp = dGU W_gu                       A K-major, B MN-major,          row tiles
-  kWgrad = 4,   // dW[e] += P_e^T Q_e                   A MN-major, B MN-major,         ragged K
+  kWgrad = 4,   // dW[e] (+)= P_e^T Q_e                 A MN-major, B MN-major,         ragged K
 };
 
 struct GemmParams {
@@ -41,22 +50,18 @@ struct GemmParams {
   int layer_stride_rows;        // wgrad
   int Mdim, Ndim, Kdim;         // wgrad: dW is [Mdim, Ndim]; row tiles: output columns, contraction
   int f;                        // expert width (fwd1 / dgrad1 addressing)
-  __nv_bfloat16* out0;          // fwd1: GU; fwd2: Yp; dgrad1: dGU; dgrad2: dXp
-  __nv_bfloat16* out1;          // fwd1: A
-  const __nv_bfloat16* GU;      // dgrad1
-  float* dW;                    // wgrad
+  int overwrite;                // wgrad: 1 = dW is written, 0 = dW is added to
   int32_t* status;
 };
 
-template <int BN> struct SmemLayout {
-  static constexpr uint32_t kBBytes = BN * BK * 2;
-  static constexpr uint32_t kStageBytes = kABytes + kBBytes;
-  static constexpr int kStages = BN == 256 ? 4 : 6;
-  static constexpr uint32_t kBarOffset = kStages * kStageBytes;
-  static constexpr uint32_t kTotal = kBarOffset + 256 + 1024;   // + barriers + alignment slack
-};
-
+// Shared memory: kStages operand stages, then one staging region per epilogue warp.
+// The SwiGLU-derivative epilogue also reads G and U, so it trades one operand stage
+// for a ring of five (G, U) chunk buffers per warp that are fetched three chunks ahead.
 template <int MODE> struct Traits {
+  static constexpr int kStages = MODE == 2 ? 3 : 4;
+  static constexpr uint32_t kStagingOffset = kStages * kStageBytes;
+  static constexpr uint32_t kStagingPerWarp = MODE == 2 ? 20480 : 8192;
+  static_assert(kStagingOffset + kEpiWarps * kStagingPerWarp == kBarOffset, "shared-memory budget");
   static constexpr bool kAMn = MODE == kWgrad;
   static constexpr bool kBMn = MODE == kDgrad1 || MODE == kDgrad2 || MODE == kWgrad;
   static constexpr bool kRowTiles = MODE != kWgrad;
@@ -64,7 +69,7 @@ template <int MODE> struct Traits {
 
 struct TileCoord { int e, mt, nt, kblocks; bool valid; };
 
-template <int MODE, int BN>
+template <int MODE>
 __device__ __forceinline__ int tiles_total(const GemmParams& p, int& n_nt, int& n_mt) {
   if constexpr (Traits<MODE>::kRowTiles) {
     n_mt = *p.offsets / BM;
@@ -117,19 +122,34 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// 32 consecutive bf16 of one row -> global (64 bytes, four 16-byte stores)
-__device__ __forceinline__ void store_row32(__nv_bfloat16* dst, const float (&v)[32]) {
-  uint4* d4 = reinterpret_cast<uint4*>(dst);
+// logistic function through one special-function op: sig(a) = 0.5 + 0.5 tanh(a/2)
+__device__ __forceinline__ float sigmoid_fast(float a) {
+  float t;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(0.5f * a));
+  return fmaf(0.5f, t, 0.5f);
+}
+
+// Staging tiles are 32 rows (one per lane) of kChunk columns in the layout the TMA
+// swizzle modes expect, so that a warp's 16-byte accesses never collide on a bank:
+//   bf16: 64-byte rows, 16-byte piece q of row r sits at piece q ^ ((r >> 1) & 3)
+//   fp32: 128-byte rows, piece q of row r sits at piece q ^ (r & 7)
+__device__ __forceinline__ uint4* bf16_piece(uint8_t* tile, int r, int q) {
+  return reinterpret_cast<uint4*>(tile + r * 64 + ((q ^ ((r >> 1) & 3)) << 4));
+}
+__device__ __forceinline__ uint4* f32_piece(uint8_t* tile, int r, int q) {
+  return reinterpret_cast<uint4*>(tile + r * 128 + ((q ^ (r & 7)) << 4));
+}
+__device__ __forceinline__ void stage_row_bf16(uint8_t* tile, int r, const float (&v)[32]) {
 #pragma unroll
   for (int q = 0; q < 4; ++q)
-    d4[q] = make_uint4(pack_bf16(v[8 * q + 0], v[8 * q + 1]), pack_bf16(v[8 * q + 2], v[8 * q + 3]),
-                       pack_bf16(v[8 * q + 4], v[8 * q + 5]), pack_bf16(v[8 * q + 6], v[8 * q + 7]));
+    *bf16_piece(tile, r, q) =
+        make_uint4(pack_bf16(v[8 * q + 0], v[8 * q + 1]), pack_bf16(v[8 * q + 2], v[8 * q + 3]),
+                   pack_bf16(v[8 * q + 4], v[8 * q + 5]), pack_bf16(v[8 * q + 6], v[8 * q + 7]));
 }
-__device__ __forceinline__ void load_row32(const __nv_bfloat16* src, float (&v)[32]) {
-  const uint4* s4 = reinterpret_cast<const uint4*>(src);
+__device__ __forceinline__ void unstage_row_bf16(uint8_t* tile, int r, float (&v)[32]) {
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
-    const uint4 w = __ldg(s4 + q);
+    const uint4 w = *bf16_piece(tile, r, q);
     const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -139,33 +159,37 @@ __device__ __forceinline__ void load_row32(const __nv_bfloat16* src, float (&v)[
   }
 }
 
-template <int MODE, int BN>
+template <int MODE>
 __global__ void __launch_bounds__(kThreads, 1)
 grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                       const __grid_constant__ CUtensorMap tmC0, const __grid_constant__ CUtensorMap tmC1,
                        const GemmParams p) {
-  using L = SmemLayout<BN>;
   using TR = Traits<MODE>;
-  constexpr int kStages = L::kStages;
+  constexpr int kStages = TR::kStages;
   constexpr uint32_t kTmemCols = 2 * BN;            // two accumulators of BN fp32 columns
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + L::kBarOffset);
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + kBarOffset);
   uint64_t* empty_bar = full_bar + kStages;
   uint64_t* tmem_full = empty_bar + kStages;
   uint64_t* tmem_empty = tmem_full + 2;
-  uint32_t* tmem_ptr = reinterpret_cast<uint32_t*>(tmem_empty + 2);
+  uint64_t* epi_bar = tmem_empty + 2;               // [kEpiWarps][5] operand loads of the epilogue
+  uint32_t* tmem_ptr = reinterpret_cast<uint32_t*>(epi_bar + 5 * kEpiWarps);
   volatile int* abort = reinterpret_cast<volatile int*>(tmem_ptr + 1);
 
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { tc::mbar_init(&full_bar[s], 1); tc::mbar_init(&empty_bar[s], 1); }
-    for (int a = 0; a < 2; ++a) { tc::mbar_init(&tmem_full[a], 1); tc::mbar_init(&tmem_empty[a], 4); }
+    for (int a = 0; a < 2; ++a) { tc::mbar_init(&tmem_full[a], 1); tc::mbar_init(&tmem_empty[a], kEpiWarps); }
+    for (int i = 0; i < 5 * kEpiWarps; ++i) tc::mbar_init(&epi_bar[i], 1);
     *abort = 0;
     tc::fence_barrier_init();
     tc::tma_prefetch_desc(&tmA);
     tc::tma_prefetch_desc(&tmB);
+    tc::tma_prefetch_desc(&tmC0);
+    if constexpr (MODE == kFwd1 || MODE == kDgrad1) tc::tma_prefetch_desc(&tmC1);
   }
   if (warp == 1) {
     tc::tmem_alloc(tmem_ptr, kTmemCols);
@@ -177,7 +201,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
   const uint32_t tmem_base = *tmem_ptr;
 
   int n_nt, n_mt;
-  const int total = tiles_total<MODE, BN>(p, n_nt, n_mt);
+  const int total = tiles_total<MODE>(p, n_nt, n_mt);
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
@@ -196,9 +220,9 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
         }
         for (int kb = 0; kb < c.kblocks; ++kb) {
           if (!tc::mbar_wait(&empty_bar[stage], phase ^ 1u, abort)) { report_timeout(p, abort, 1); ok = false; break; }
-          uint8_t* sA = smem + stage * L::kStageBytes;
+          uint8_t* sA = smem + stage * kStageBytes;
           uint8_t* sB = sA + kABytes;
-          tc::mbar_expect_tx(&full_bar[stage], L::kStageBytes);
+          tc::mbar_expect_tx(&full_bar[stage], kStageBytes);
           if constexpr (MODE == kFwd1) {
             tc::tma_load_2d(sA, &tmA, &full_bar[stage], kb * BK, c.mt * BM);
             tc::tma_load_3d(sB, &tmB, &full_bar[stage], kb * BK, c.nt * (BN / 2), 2 * pe);
@@ -258,7 +282,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
         for (int kb = 0; kb < c.kblocks; ++kb) {
           if (!tc::mbar_wait(&full_bar[stage], phase, abort)) { report_timeout(p, abort, 3); ok = false; break; }
           tc::tc_fence_after_sync();
-          const uint32_t aaddr = tc::smem_u32(smem + stage * L::kStageBytes);
+          const uint32_t aaddr = tc::smem_u32(smem + stage * kStageBytes);
           const uint64_t adesc = tc::smem_desc_sw128(aaddr, a_lbo, 1024);
           const uint64_t bdesc = tc::smem_desc_sw128(aaddr + kABytes, b_lbo, 1024);
 #pragma unroll
@@ -272,101 +296,189 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     }
   } else {
     // ------------------------------------------------------------ epilogue (warps 2..5)
-    const int quarter = warp & 3;                        // TMEM lanes [32*quarter, 32*quarter + 32)
+    // Warp w owns TMEM lanes [32*(w%4), +32) = 32 rows of the tile.  Results are rounded,
+    // staged in this warp's shared-memory tiles and leave through TMA stores; nothing
+    // here synchronises with another warp except the two TMEM barriers.
+    const int quarter = warp & 3;
+    const int ew = warp - 2;
+    uint8_t* stg = smem + TR::kStagingOffset + ew * TR::kStagingPerWarp;
+    constexpr int kRing = 5, kAhead = 3;               // dgrad1: (G, U) chunk buffers, prefetch distance
+    uint64_t* my_bar = epi_bar + kRing * ew;
+    int gchunk = 0;                                    // chunks this warp has staged so far (ring position)
+    (void)my_bar;
     int local = 0;
-    for (int tile = blockIdx.x; tile < total; tile += gridDim.x) {
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
       const TileCoord c = tile_coord<MODE>(p, tile, n_nt, n_mt);
-      if (!c.valid) continue;
+      if (!c.valid) {
+        if constexpr (MODE == kWgrad) {
+          if (p.overwrite) {                           // no rows anywhere: the gradient of this tile is zero
+            const int m0 = c.mt * BM + quarter * 32;
+            if (m0 < p.Mdim) {
+              if (lane == 0) tc::bulk_wait_read<0>();
+              __syncwarp();
+#pragma unroll
+              for (int q = 0; q < 8; ++q) *f32_piece(stg, lane, q) = make_uint4(0, 0, 0, 0);
+              tc::fence_proxy_async();
+              __syncwarp();
+              if (lane == 0) {
+                for (int ch = 0; ch < BN / kChunk; ++ch) {
+                  const int col = c.nt * BN + ch * kChunk;
+                  if (col < p.Ndim) tc::tma_store_2d(&tmC0, stg, col, (p.expert_base + c.e) * p.Mdim + m0);
+                }
+                tc::bulk_commit();
+                tc::bulk_wait_read<0>();
+              }
+              __syncwarp();
+            }
+          }
+        }
+        continue;
+      }
       const int acc = local & 1;
       const uint32_t acc_phase = (local >> 1) & 1;
       ++local;
+      const int row0 = c.mt * BM + quarter * 32;       // first row of this warp (row tiles: permuted row)
+
+      // dgrad1: chunk j of this tile (global chunk gchunk + j) lands in ring slot (gchunk + j) % kRing.
+      // A slot is refilled only after the store that last read it has drained: that store is
+      // at least two bulk groups old whenever a fetch is issued, hence wait_group.read 1.
+      int nch = 0;
+      auto fetch_gu = [&](int j) {
+        const int slot = (gchunk + j) % kRing;
+        uint8_t* buf = stg + slot * 2 * kBf16ChunkBytes;
+        const int col = c.nt * BN + j * kChunk;
+        tc::bulk_wait_read<1>();
+        tc::mbar_expect_tx(&my_bar[slot], 2 * kBf16ChunkBytes);
+        tc::tma_load_2d(buf, &tmC1, &my_bar[slot], col, row0);
+        tc::tma_load_2d(buf + kBf16ChunkBytes, &tmC1, &my_bar[slot], p.f + col, row0);
+      };
+      if constexpr (MODE == kDgrad1) {                 // fetch the first chunks while the MMAs still run
+        nch = min(BN / kChunk, (p.f - c.nt * BN) / kChunk);
+        if (lane == 0)
+          for (int j = 0; j < kAhead && j < nch; ++j) fetch_gu(j);
+      }
       if (!tc::mbar_wait(&tmem_full[acc], acc_phase, abort)) {
         if (lane == 0) report_timeout(p, abort, 4);
         break;
       }
       tc::tc_fence_after_sync();
       const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * BN;
-      const int row_in_tile = quarter * 32 + lane;
 
       if constexpr (MODE == kFwd1) {
-        const int64_t row = (int64_t)c.mt * BM + row_in_tile;
-        const int feat0 = c.nt * (BN / 2);
 #pragma unroll 1
-        for (int ch = 0; ch < BN / 64; ++ch) {
+        for (int ch = 0; ch < BN / 2 / kChunk; ++ch) {
+          const int feat = c.nt * (BN / 2) + ch * kChunk;
+          if (feat >= p.f) break;
           uint32_t rg[32], ru[32];
-          tc::tmem_ld_32x32(t_row + ch * 32, rg);
-          tc::tmem_ld_32x32(t_row + BN / 2 + ch * 32, ru);
+          tc::tmem_ld_32x32(t_row + ch * kChunk, rg);
+          tc::tmem_ld_32x32(t_row + BN / 2 + ch * kChunk, ru);
           tc::tmem_ld_wait();
-          const int feat = feat0 + ch * 32;
-          if (feat < p.f) {
-            float g[32], u[32], a[32];
+          float g[32], u[32], a[32];
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              g[i] = __uint_as_float(rg[i]);
-              u[i] = __uint_as_float(ru[i]);
-              a[i] = silu_f(g[i]) * u[i];
-            }
-            store_row32(p.out0 + row * 2 * p.f + feat, g);
-            store_row32(p.out0 + row * 2 * p.f + p.f + feat, u);
-            store_row32(p.out1 + row * p.f + feat, a);
+          for (int i = 0; i < 32; ++i) {
+            g[i] = __uint_as_float(rg[i]);
+            u[i] = __uint_as_float(ru[i]);
+            a[i] = g[i] * sigmoid_fast(g[i]) * u[i];
+          }
+          if (lane == 0) tc::bulk_wait_read<0>();      // the previous chunk's stores have drained the tiles
+          __syncwarp();
+          stage_row_bf16(stg, lane, g);
+          stage_row_bf16(stg + kBf16ChunkBytes, lane, u);
+          stage_row_bf16(stg + 2 * kBf16ChunkBytes, lane, a);
+          tc::fence_proxy_async();
+          __syncwarp();
+          if (lane == 0) {
+            tc::tma_store_2d(&tmC0, stg, feat, row0);
+            tc::tma_store_2d(&tmC0, stg + kBf16ChunkBytes, p.f + feat, row0);
+            tc::tma_store_2d(&tmC1, stg + 2 * kBf16ChunkBytes, feat, row0);
+            tc::bulk_commit();
           }
         }
       } else if constexpr (MODE == kFwd2 || MODE == kDgrad2) {
-        const int64_t row = (int64_t)c.mt * BM + row_in_tile;
 #pragma unroll 1
-        for (int ch = 0; ch < BN / 32; ++ch) {
+        for (int ch = 0; ch < BN / kChunk; ++ch) {
+          const int col = c.nt * BN + ch * kChunk;
+          if (col >= p.Ndim) break;
           uint32_t rr[32];
-          tc::tmem_ld_32x32(t_row + ch * 32, rr);
+          tc::tmem_ld_32x32(t_row + ch * kChunk, rr);
           tc::tmem_ld_wait();
-          const int col = c.nt * BN + ch * 32;
-          if (col < p.Ndim) {
-            float v[32];
+          float v[32];
 #pragma unroll
-            for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(rr[i]);
-            store_row32(p.out0 + row * p.Ndim + col, v);
+          for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(rr[i]);
+          uint8_t* buf = stg + (gchunk++ & 3) * kBf16ChunkBytes;
+          if (lane == 0) tc::bulk_wait_read<3>();      // the store issued four chunks ago has drained `buf`
+          __syncwarp();
+          stage_row_bf16(buf, lane, v);
+          tc::fence_proxy_async();
+          __syncwarp();
+          if (lane == 0) {
+            tc::tma_store_2d(&tmC0, buf, col, row0);
+            tc::bulk_commit();
           }
         }
       } else if constexpr (MODE == kDgrad1) {
-        const int64_t row = (int64_t)c.mt * BM + row_in_tile;
 #pragma unroll 1
-        for (int ch = 0; ch < BN / 32; ++ch) {
+        for (int ch = 0; ch < nch; ++ch) {
+          const int col = c.nt * BN + ch * kChunk;
+          const int slot = (gchunk + ch) % kRing;
+          const uint32_t slot_phase = ((gchunk + ch) / kRing) & 1;
+          uint8_t* buf = stg + slot * 2 * kBf16ChunkBytes;
+          if (lane == 0 && ch + kAhead < nch) fetch_gu(ch + kAhead);
           uint32_t rr[32];
-          tc::tmem_ld_32x32(t_row + ch * 32, rr);
+          tc::tmem_ld_32x32(t_row + ch * kChunk, rr);
           tc::tmem_ld_wait();
-          const int col = c.nt * BN + ch * 32;
-          if (col < p.f) {
-            float g[32], u[32], dg[32], du[32];
-            load_row32(p.GU + row * 2 * p.f + col, g);
-            load_row32(p.GU + row * 2 * p.f + p.f + col, u);
+          if (!tc::mbar_wait(&my_bar[slot], slot_phase, abort)) {
+            if (lane == 0) report_timeout(p, abort, 5);
+            ok = false;
+            break;
+          }
+          float g[32], u[32], dg[32], du[32];
+          unstage_row_bf16(buf, lane, g);
+          unstage_row_bf16(buf + kBf16ChunkBytes, lane, u);
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              const float dA = __uint_as_float(rr[i]);
-              dg[i] = dA * u[i] * silu_grad_f(g[i]);
-              du[i] = dA * silu_f(g[i]);
-            }
-            store_row32(p.out0 + row * 2 * p.f + col, dg);
-            store_row32(p.out0 + row * 2 * p.f + p.f + col, du);
+          for (int i = 0; i < 32; ++i) {
+            const float dA = __uint_as_float(rr[i]);
+            const float sig = sigmoid_fast(g[i]);
+            const float sl = g[i] * sig;
+            dg[i] = dA * u[i] * (sig + sl * (1.0f - sig));   // silu'(g) = sig (1 + g (1 - sig))
+            du[i] = dA * sl;
+          }
+          stage_row_bf16(buf, lane, dg);               // in place: each lane rewrites the row it read
+          stage_row_bf16(buf + kBf16ChunkBytes, lane, du);
+          tc::fence_proxy_async();
+          __syncwarp();
+          if (lane == 0) {
+            tc::tma_store_2d(&tmC0, buf, col, row0);
+            tc::tma_store_2d(&tmC0, buf + kBf16ChunkBytes, p.f + col, row0);
+            tc::bulk_commit();
           }
         }
+        gchunk += nch;
+        if (!ok) break;
       } else {
-        const int m = c.mt * BM + row_in_tile;
-        float* out = p.dW + ((int64_t)(p.expert_base + c.e) * p.Mdim + m) * p.Ndim;
+        const int m0 = row0;                           // row of dW[e]
+        if (m0 < p.Mdim) {
+          const int grow = (p.expert_base + c.e) * p.Mdim + m0;
 #pragma unroll 1
-        for (int ch = 0; ch < BN / 32; ++ch) {
-          uint32_t rr[32];
-          tc::tmem_ld_32x32(t_row + ch * 32, rr);
-          tc::tmem_ld_wait();
-          const int col = c.nt * BN + ch * 32;
-          if (m < p.Mdim && col < p.Ndim) {
-            float4* o4 = reinterpret_cast<float4*>(out + col);
+          for (int ch = 0; ch < BN / kChunk; ++ch) {
+            const int col = c.nt * BN + ch * kChunk;
+            if (col >= p.Ndim) break;
+            uint32_t rr[32];
+            tc::tmem_ld_32x32(t_row + ch * kChunk, rr);
+            tc::tmem_ld_wait();
+            uint8_t* buf = stg + (gchunk++ & 1) * kF32ChunkBytes;
+            if (lane == 0) tc::bulk_wait_read<1>();    // the store issued two chunks ago has drained `buf`
+            __syncwarp();
 #pragma unroll
-            for (int q = 0; q < 8; ++q) {
-              float4 cur = o4[q];
-              cur.x += __uint_as_float(rr[4 * q + 0]);
-              cur.y += __uint_as_float(rr[4 * q + 1]);
-              cur.z += __uint_as_float(rr[4 * q + 2]);
-              cur.w += __uint_as_float(rr[4 * q + 3]);
-              o4[q] = cur;
+            for (int q = 0; q < 8; ++q)
+              *f32_piece(buf, lane, q) = make_uint4(rr[4 * q + 0], rr[4 * q + 1], rr[4 * q + 2], rr[4 * q + 3]);
+            tc::fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) {
+              if (p.overwrite) tc::tma_store_2d(&tmC0, buf, col, grow);
+              else tc::tma_reduce_add_2d(&tmC0, buf, col, grow);
+              tc::bulk_commit();
             }
           }
         }
@@ -375,6 +487,10 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
       __syncwarp();
       if (lane == 0) tc::mbar_arrive(&tmem_empty[acc]);
     }
+    if (!ok && lane == 0)
+      for (int i = 0; i < 200; ++i) __nanosleep(1000);  // let loads already in flight land before the CTA retires
+    if (lane == 0) tc::bulk_wait<0>();                 // every store has left shared memory and is complete
+    __syncwarp();
   }
 
   tc::tc_fence_before_sync();
@@ -394,44 +510,57 @@ struct TcModule {
   EncodeTiledFn encode;
 };
 
-// bf16 tensor map with the 128-byte swizzle; dims/box innermost first, strides in elements.
-int make_tmap(const unipool_ctx* ctx, CUtensorMap* out, const void* base, int rank, const uint64_t* dims,
-              const uint64_t* strides_elems, const uint32_t* box) {
+enum MapKind { kMapOperand, kMapBf16Chunk, kMapF32Chunk };
+
+// Tensor map over a dense row-major tensor; dims/box innermost first, strides in elements.
+//   kMapOperand   bf16, 128-byte swizzle (MMA operand tiles)
+//   kMapBf16Chunk bf16, 64-byte swizzle  (32 x 32 epilogue chunks)
+//   kMapF32Chunk  fp32, 128-byte swizzle (32 x 32 epilogue chunks of the weight gradient)
+int make_tmap(const unipool_ctx* ctx, CUtensorMap* out, MapKind kind, const void* base, int rank,
+              const uint64_t* dims, const uint64_t* strides_elems, const uint32_t* box) {
   const TcModule* mod = static_cast<const TcModule*>(ctx->tmap_cache);
+  const uint64_t esz = kind == kMapF32Chunk ? 4 : 2;
   cuuint64_t gdims[3], gstrides[2];
   cuuint32_t gbox[3], estr[3] = {1, 1, 1};
   for (int i = 0; i < rank; ++i) { gdims[i] = dims[i]; gbox[i] = box[i]; }
-  for (int i = 0; i + 1 < rank; ++i) gstrides[i] = strides_elems[i] * 2;
+  for (int i = 0; i + 1 < rank; ++i) gstrides[i] = strides_elems[i] * esz;
   UP_REQUIRE((reinterpret_cast<uintptr_t>(base) & 15) == 0, UNIPOOL_ERR_INVALID_ARG,
              "tensor base %p is not 16-byte aligned", base);
-  CUresult r = mod->encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gdims,
-                           gstrides, gbox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+  CUresult r = mod->encode(out, kind == kMapF32Chunk ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
+                           (cuuint32_t)rank, const_cast<void*>(base), gdims, gstrides, gbox, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE,
+                           kind == kMapBf16Chunk ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   UP_REQUIRE(r == CUDA_SUCCESS, UNIPOOL_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
   return UNIPOOL_OK;
 }
 
 int map_2d(const unipool_ctx* ctx, CUtensorMap* out, const void* base, uint64_t cols, uint64_t rows,
-           uint32_t box_cols, uint32_t box_rows) {
+           uint32_t box_cols, uint32_t box_rows, MapKind kind = kMapOperand) {
   const uint64_t dims[2] = {cols, rows}, strides[1] = {cols};
   const uint32_t box[2] = {box_cols, box_rows};
-  return make_tmap(ctx, out, base, 2, dims, strides, box);
+  return make_tmap(ctx, out, kind, base, 2, dims, strides, box);
 }
 
-template <int MODE, int BN>
-int launch(unipool_ctx* ctx, int phase, const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmParams& p,
-           cudaStream_t s) {
+// 32 x 32 epilogue chunk map
+int map_chunk(const unipool_ctx* ctx, CUtensorMap* out, const void* base, uint64_t cols, uint64_t rows,
+              MapKind kind) {
+  return map_2d(ctx, out, base, cols, rows, kChunk, 32, kind);
+}
+
+template <int MODE>
+int launch(unipool_ctx* ctx, int phase, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC0,
+           const CUtensorMap& tmC1, const GemmParams& p, cudaStream_t s) {
   PhaseTimer pt(ctx, phase, 1, s);
-  auto kern = grouped_gemm_tc_kernel<MODE, BN>;
-  constexpr int smem = SmemLayout<BN>::kTotal;
-  UP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-  kern<<<ctx->sm_count, kThreads, smem, s>>>(tmA, tmB, p);
+  auto kern = grouped_gemm_tc_kernel<MODE>;
+  UP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemTotal));
+  kern<<<ctx->sm_count, kThreads, kSmemTotal, s>>>(tmA, tmB, tmC0, tmC1, p);
   UP_LAUNCH_CHECK();
   return UNIPOOL_OK;
 }
 
 int wgrad_pair(unipool_ctx* ctx, const PoolWgradArgs& a, cudaStream_t s) {
-  const int d = ctx->cfg.d_model, f = ctx->cfg.d_ff;
+  const int d = ctx->cfg.d_model, f = ctx->cfg.d_ff, M = ctx->cfg.pool_size;
   const uint64_t rows = (uint64_t)(a.n_layers > 1 ? (int64_t)a.n_layers * a.layer_stride_rows : ctx->row_capacity);
   GemmParams p{};
   p.offsets = a.offsets;
@@ -439,19 +568,22 @@ int wgrad_pair(unipool_ctx* ctx, const PoolWgradArgs& a, cudaStream_t s) {
   p.expert_base = a.expert_base;
   p.n_layers = a.n_layers;
   p.layer_stride_rows = (int)a.layer_stride_rows;
+  p.overwrite = a.overwrite ? 1 : 0;
   p.status = ctx->ws.status;
-  CUtensorMap tmP, tmQ;
+  CUtensorMap tmP, tmQ, tmW;
   int rc;
-  // dW_down[e] [d, f] += dYp_e^T A_e
+  // dW_down[e] [d, f] (+)= dYp_e^T A_e
   if ((rc = map_2d(ctx, &tmP, a.dYp, d, rows, 64, 64)) != UNIPOOL_OK) return rc;
   if ((rc = map_2d(ctx, &tmQ, a.A, f, rows, 64, 64)) != UNIPOOL_OK) return rc;
-  p.Mdim = d; p.Ndim = f; p.dW = a.dW_down;
-  if ((rc = launch<kWgrad, 128>(ctx, UNIPOOL_PH_WGRAD_DOWN, tmP, tmQ, p, s)) != UNIPOOL_OK) return rc;
-  // dW_gu[e] [2f, d] += dGU_e^T Xp_e
+  if ((rc = map_chunk(ctx, &tmW, a.dW_down, f, (uint64_t)M * d, kMapF32Chunk)) != UNIPOOL_OK) return rc;
+  p.Mdim = d; p.Ndim = f;
+  if ((rc = launch<kWgrad>(ctx, UNIPOOL_PH_WGRAD_DOWN, tmP, tmQ, tmW, tmW, p, s)) != UNIPOOL_OK) return rc;
+  // dW_gu[e] [2f, d] (+)= dGU_e^T Xp_e
   if ((rc = map_2d(ctx, &tmP, a.dGU, 2 * f, rows, 64, 64)) != UNIPOOL_OK) return rc;
   if ((rc = map_2d(ctx, &tmQ, a.Xp, d, rows, 64, 64)) != UNIPOOL_OK) return rc;
-  p.Mdim = 2 * f; p.Ndim = d; p.dW = a.dW_gu;
-  return launch<kWgrad, 128>(ctx, UNIPOOL_PH_WGRAD_GU, tmP, tmQ, p, s);
+  if ((rc = map_chunk(ctx, &tmW, a.dW_gu, d, (uint64_t)M * 2 * f, kMapF32Chunk)) != UNIPOOL_OK) return rc;
+  p.Mdim = 2 * f; p.Ndim = d;
+  return launch<kWgrad>(ctx, UNIPOOL_PH_WGRAD_GU, tmP, tmQ, tmW, tmW, p, s);
 }
 
 }  // namespace
@@ -482,28 +614,27 @@ int expert_fwd_tc(unipool_ctx* ctx, const ExpertFwdArgs& a, cudaStream_t s) {
   p.expert_base = a.expert_base;
   p.f = f;
   p.status = ctx->ws.status;
-  CUtensorMap tmA, tmB;
+  CUtensorMap tmA, tmB, tmC0, tmC1;
   int rc;
-  // GU = Xp [W_gate; W_up]^T with the SwiGLU epilogue.  B tile = 64 gate rows + 64 up rows of the
+  // GU = Xp [W_gate; W_up]^T with the SwiGLU epilogue.  B tile = 128 gate rows + 128 up rows of the
   // same features, fetched as one 3-D box over W_gu viewed as [2M, f, d].
-  if ((rc = map_2d(ctx, &tmA, a.Xp, d, cap, 64, 128)) != UNIPOOL_OK) return rc;
+  if ((rc = map_2d(ctx, &tmA, a.Xp, d, cap, 64, BM)) != UNIPOOL_OK) return rc;
   {
     const uint64_t dims[3] = {(uint64_t)d, (uint64_t)f, (uint64_t)2 * M};
     const uint64_t strides[2] = {(uint64_t)d, (uint64_t)f * d};
-    const uint32_t box[3] = {64, 64, 2};
-    if ((rc = make_tmap(ctx, &tmB, a.W_gu, 3, dims, strides, box)) != UNIPOOL_OK) return rc;
+    const uint32_t box[3] = {64, BN / 2, 2};
+    if ((rc = make_tmap(ctx, &tmB, kMapOperand, a.W_gu, 3, dims, strides, box)) != UNIPOOL_OK) return rc;
   }
+  if ((rc = map_chunk(ctx, &tmC0, a.GU, 2 * f, cap, kMapBf16Chunk)) != UNIPOOL_OK) return rc;
+  if ((rc = map_chunk(ctx, &tmC1, a.A, f, cap, kMapBf16Chunk)) != UNIPOOL_OK) return rc;
   p.Ndim = f; p.Kdim = d;
-  p.out0 = static_cast<__nv_bfloat16*>(a.GU);
-  p.out1 = static_cast<__nv_bfloat16*>(a.A);
-  if ((rc = launch<kFwd1, 128>(ctx, UNIPOOL_PH_EXPERT_FWD_GU, tmA, tmB, p, s)) != UNIPOOL_OK) return rc;
+  if ((rc = launch<kFwd1>(ctx, UNIPOOL_PH_EXPERT_FWD_GU, tmA, tmB, tmC0, tmC1, p, s)) != UNIPOOL_OK) return rc;
   // Yp = A W_down^T
-  if ((rc = map_2d(ctx, &tmA, a.A, f, cap, 64, 128)) != UNIPOOL_OK) return rc;
-  if ((rc = map_2d(ctx, &tmB, a.W_down, f, (uint64_t)M * d, 64, 128)) != UNIPOOL_OK) return rc;
+  if ((rc = map_2d(ctx, &tmA, a.A, f, cap, 64, BM)) != UNIPOOL_OK) return rc;
+  if ((rc = map_2d(ctx, &tmB, a.W_down, f, (uint64_t)M * d, 64, BN)) != UNIPOOL_OK) return rc;
+  if ((rc = map_chunk(ctx, &tmC0, a.Yp, d, cap, kMapBf16Chunk)) != UNIPOOL_OK) return rc;
   p.Ndim = d; p.Kdim = f;
-  p.out0 = static_cast<__nv_bfloat16*>(a.Yp);
-  p.out1 = nullptr;
-  return launch<kFwd2, 128>(ctx, UNIPOOL_PH_EXPERT_FWD_DOWN, tmA, tmB, p, s);
+  return launch<kFwd2>(ctx, UNIPOOL_PH_EXPERT_FWD_DOWN, tmA, tmB, tmC0, tmC0, p, s);
 }
 
 int expert_bwd_tc(unipool_ctx* ctx, const ExpertBwdArgs& a, cudaStream_t s) {
@@ -516,23 +647,24 @@ int expert_bwd_tc(unipool_ctx* ctx, const ExpertBwdArgs& a, cudaStream_t s) {
   p.expert_base = a.expert_base;
   p.f = f;
   p.status = ctx->ws.status;
-  CUtensorMap tmA, tmB;
+  CUtensorMap tmA, tmB, tmC0, tmC1;
   int rc;
   // dA = dYp W_down, fused with the SwiGLU derivative -> dGU
-  if ((rc = map_2d(ctx, &tmA, a.dYp, d, cap, 64, 128)) != UNIPOOL_OK) return rc;
+  if ((rc = map_2d(ctx, &tmA, a.dYp, d, cap, 64, BM)) != UNIPOOL_OK) return rc;
   if ((rc = map_2d(ctx, &tmB, a.W_down, f, (uint64_t)M * d, 64, 64)) != UNIPOOL_OK) return rc;
+  if ((rc = map_chunk(ctx, &tmC0, a.dGU, 2 * f, cap, kMapBf16Chunk)) != UNIPOOL_OK) return rc;
+  if ((rc = map_chunk(ctx, &tmC1, a.GU, 2 * f, cap, kMapBf16Chunk)) != UNIPOOL_OK) return rc;
   p.Ndim = f; p.Kdim = d;
-  p.GU = static_cast<const __nv_bfloat16*>(a.GU);
-  p.out0 = static_cast<__nv_bfloat16*>(a.dGU);
-  if ((rc = launch<kDgrad1, 128>(ctx, UNIPOOL_PH_DGRAD_DOWN, tmA, tmB, p, s)) != UNIPOOL_OK) return rc;
+  if ((rc = launch<kDgrad1>(ctx, UNIPOOL_PH_DGRAD_DOWN, tmA, tmB, tmC0, tmC1, p, s)) != UNIPOOL_OK) return rc;
   // dXp = dGU [W_gate; W_up]
-  if ((rc = map_2d(ctx, &tmA, a.dGU, 2 * f, cap, 64, 128)) != UNIPOOL_OK) return rc;
+  if ((rc = map_2d(ctx, &tmA, a.dGU, 2 * f, cap, 64, BM)) != UNIPOOL_OK) return rc;
   if ((rc = map_2d(ctx, &tmB, a.W_gu, d, (uint64_t)M * 2 * f, 64, 64)) != UNIPOOL_OK) return rc;
+  if ((rc = map_chunk(ctx, &tmC0, a.dXp, d, cap, kMapBf16Chunk)) != UNIPOOL_OK) return rc;
   p.Ndim = d; p.Kdim = 2 * f;
-  p.out0 = static_cast<__nv_bfloat16*>(a.dXp);
-  if ((rc = launch<kDgrad2, 128>(ctx, UNIPOOL_PH_DGRAD_GU, tmA, tmB, p, s)) != UNIPOOL_OK) return rc;
+  if ((rc = launch<kDgrad2>(ctx, UNIPOOL_PH_DGRAD_GU, tmA, tmB, tmC0, tmC0, p, s)) != UNIPOOL_OK) return rc;
   if (a.wgrad) {
-    PoolWgradArgs w{1, 0, a.offsets, a.Xp, a.A, a.dYp, a.dGU, a.expert_base, a.n_experts, a.dW_gu, a.dW_down};
+    PoolWgradArgs w{1, 0, a.offsets, a.Xp, a.A, a.dYp, a.dGU, a.expert_base, a.n_experts, a.dW_gu, a.dW_down,
+                    a.overwrite};
     return wgrad_pair(ctx, w, s);
   }
   return UNIPOOL_OK;

@@ -96,6 +96,9 @@ class UniPoolStack:
     def zero_grad(self):
         self.dW_gu.zero_(); self.dW_down.zero_(); self.dW_r.zero_(); self.dsigma.zero_()
 
+    def zero_router_grad(self):
+        self.dW_r.zero_(); self.dsigma.zero_()
+
     # ------------------------------------------------------------------ forward
     def forward_layer(self, l, T=None):
         T = self.T if T is None else T
@@ -130,11 +133,13 @@ class UniPoolStack:
         return self.loss
 
     # ------------------------------------------------------------------ backward
-    def backward_layer(self, l, dx_next, dx_out, T=None, with_aux=True):
+    def backward_layer(self, l, dx_next, dx_out, T=None, with_aux=True, overwrite=False):
+        """``overwrite``: this layer's weight gradient replaces what the pool-gradient
+        slices of its view hold (the first contribution of a step) instead of adding to it."""
         T = self.T if T is None else T
         c = self.ctx
         s = l if self.deferred_wgrad else 0
-        flags = B.BWD_SKIP_WGRAD if self.deferred_wgrad else 0
+        flags = B.BWD_SKIP_WGRAD if self.deferred_wgrad else (B.WGRAD_OVERWRITE if overwrite else 0)
         c.expert_bwd(dx_next, T, self.row_of[l], self.gate[l], self.token_of[l], self.offsets[l],
                      self.tile_expert[l], self.Xp[l], self.GU[l], self.A[l], self.Yp[l], self.W_gu,
                      self.W_down, self.base(l), self.m, dx_next, self.dYp[s], self.dGU[s], dx_out,
@@ -145,24 +150,30 @@ class UniPoolStack:
         c.route_bwd(self.x[l], T, self.W_r[l], self.sigma[l], self.m, self.znorm[l], self.z[l],
                     self.idx[l], self.dgate, coef, dx_out, self.dW_r[l], self.dsigma[l:l + 1])
 
-    def backward(self, upstream=None, T=None, with_aux=True):
+    def backward(self, upstream=None, T=None, with_aux=True, accumulate=True):
+        """``accumulate=False``: the pool gradient of this pass replaces the buffers' contents
+        (the first weight-gradient contribution to each expert is a store, the rest add), so the
+        buffers need no zeroing; router gradients always add."""
         T = self.T if T is None else T
         cur = 0
         if upstream is not None:
             self.dx[cur, :T].copy_(upstream, non_blocking=True)
         for l in reversed(range(self.L)):
-            self.backward_layer(l, self.dx[cur], self.dx[1 - cur], T, with_aux)
+            first = (not accumulate) and (bool(self.private) or l == self.L - 1)
+            self.backward_layer(l, self.dx[cur], self.dx[1 - cur], T, with_aux, overwrite=first)
             cur = 1 - cur
         if self.deferred_wgrad:
             self.ctx.pool_wgrad(self.L, self.cap, self.offsets, self.Xp, self.A, self.dYp, self.dGU,
-                                0, self.m, self.dW_gu, self.dW_down)
+                                0, self.m, self.dW_gu, self.dW_down, 0 if accumulate else B.WGRAD_OVERWRITE)
         return self.dx[cur]
 
-    def step(self, x0=None, upstream=None, T=None):
+    def step(self, x0=None, upstream=None, T=None, accumulate=True):
         """One pass of the whole hot path: forward, balance loss, backward."""
         self.forward(x0, T)
         self.aux_loss(T)
-        return self.backward(upstream, T)
+        if not accumulate:
+            self.zero_router_grad()
+        return self.backward(upstream, T, accumulate=accumulate)
 
     def close(self):
         self.ctx.close()

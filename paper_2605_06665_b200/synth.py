@@ -10,7 +10,13 @@ sigma_l = 1; upstream gradient ~ N(0,1) [T,d]; one numpy PCG64 stream per tensor
 derived from (seed, tensor tag, layer).  In bf16 mode every tensor is rounded to
 a bf16-representable value once, here, and returned as float32, so that both
 sides read identical numbers.  The skewed workload adds to layer l's logits the
-bias  beta * ln p(rank_l(i)),  p(r) ~ r^-1.1 (Zipf), rank_l a seeded permutation.
+bias  beta * (ln p(rank_l(i)) - mean_j ln p(j)),  p(r) ~ r^-1.1 (Zipf), rank_l a
+seeded permutation.  The bias is centred because the NormRouter score is
+max(0, z/||z||): unlike a softmax it is not invariant to a common shift of the
+logits, and an all-negative bias would zero almost every gate.  beta = 0.4 is the
+smallest multiple of 0.05 for which, at seed 0, every layer of the skewed workload
+has at least one expert without tokens (and one expert that more than 5 % of the
+tokens select).
 """
 from __future__ import annotations
 
@@ -27,7 +33,7 @@ CONFIGS = {
     "978m":           dict(L=24, d=1536, f=4096, M=192, k=2, T=32768, dtype="bf16", private=0, zipf_beta=0.0),
     "978m_pool128":   dict(L=24, d=1536, f=4096, M=128, k=2, T=32768, dtype="bf16", private=0, zipf_beta=0.0),
     "978m_vanilla":   dict(L=24, d=1536, f=4096, M=192, k=2, T=32768, dtype="bf16", private=8, zipf_beta=0.0),
-    "fine_zipf":      dict(L=12, d=768,  f=512,  M=384, k=8, T=16384, dtype="bf16", private=0, zipf_beta=0.35),
+    "fine_zipf":      dict(L=12, d=768,  f=512,  M=384, k=8, T=16384, dtype="bf16", private=0, zipf_beta=0.4),
 }
 
 EPS = 1e-6          # "small constant for numerical stability" of Eq. 7
@@ -76,7 +82,8 @@ def zipf_bias(cfg, layer, seed=0):
     p = ranks ** (-ZIPF_S)
     p /= p.sum()
     perm = _rng(seed, 7, layer).permutation(m)          # expert i has rank perm[i]+1
-    return (beta * np.log(p[perm])).astype(np.float32)
+    logp = np.log(p)
+    return (beta * (logp[perm] - logp.mean())).astype(np.float32)
 
 
 def make_inputs(cfg, seed=0, T=None, L=None):
