@@ -220,8 +220,8 @@ def run_ours(args):
     abytes = algorithmic_bytes(cfg, st.cap)
     for name, factor in GEMM_PHASES.items():
         if name in kernels:
-            flops = factor * R * d * f
-            tf = flops / (kernels[name]["ms_per_call"] * 1e-3) / 1e12
+            flops = factor * R * d * f * L               # per step, whatever the number of launches
+            tf = flops / (kernels[name]["ms_per_step"] * 1e-3) / 1e12
             kernels[name].update(tflops=tf, frac_of_measured_sustained=tf / peaks["bf16_tflops_sustained"])
     for name, nbytes in abytes.items():
         if name in kernels:

@@ -21,10 +21,11 @@ void set_error(const char* fmt, ...) {
 
 // Debug aid: UNIPOOL_FORCE_SIMT=1 runs the bf16 grouped GEMMs on the CUDA-core path
 // (same arithmetic contract, far slower); used to bisect tensor-core issues.
-static bool use_tensor_cores(const unipool_ctx* ctx) {
+bool force_simt() {
   static const bool forced = [] { const char* v = getenv("UNIPOOL_FORCE_SIMT"); return v && v[0] == '1'; }();
-  return ctx->cfg.dtype == UNIPOOL_BF16 && !forced;
+  return forced;
 }
+static bool use_tensor_cores(const unipool_ctx* ctx) { return ctx->cfg.dtype == UNIPOOL_BF16 && !force_simt(); }
 
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -50,8 +51,14 @@ Workspace carve_workspace(const unipool_config& cfg, void* base) {
   w.route_sums = reinterpret_cast<double*>(take(UNIPOOL_MAX_EXPERTS * sizeof(double)));
   w.tickets = reinterpret_cast<uint32_t*>(take(8 * sizeof(uint32_t)));
   w.dsigma_acc = reinterpret_cast<double*>(take(2 * sizeof(double)));
+  w.split_any = reinterpret_cast<int32_t*>(take(4 * sizeof(int32_t)));
   w.block_hist = reinterpret_cast<int32_t*>(take((size_t)blocks * UNIPOOL_MAX_EXPERTS * sizeof(int32_t)));
-  w.dz = reinterpret_cast<float*>(take((size_t)cfg.max_tokens * cfg.pool_size * sizeof(float)));
+  {
+    const size_t mp = ((size_t)cfg.pool_size + 63) / 64 * 64;
+    const size_t per_token = cfg.dtype == UNIPOOL_BF16 ? mp * 2 : (size_t)cfg.pool_size * sizeof(float);
+    w.dz = reinterpret_cast<float*>(take((size_t)cfg.max_tokens * per_token));
+  }
+  w.w_split = cfg.dtype == UNIPOOL_BF16 ? take((size_t)3 * cfg.pool_size * cfg.d_model * 2) : nullptr;
   w.dXp = take((size_t)cap * cfg.d_model * eb);
   w.bytes = off;
   return w;

@@ -13,6 +13,7 @@ namespace unipool {
 
 // ---------------------------------------------------------------- errors
 void set_error(const char* fmt, ...);
+bool force_simt();   // debug aid: UNIPOOL_FORCE_SIMT=1 runs the bf16 mode on the CUDA-core kernels
 
 #define UP_REQUIRE(cond, code, ...)      \
   do {                                   \
@@ -51,7 +52,9 @@ struct Workspace {
   uint32_t* tickets;      // [8]   "last block done" counters, self-cleaning
   double*  dsigma_acc;    // [2]   self-cleaning accumulator of route_bwd / calibrate_c
   int32_t* block_hist;    // [dispatch_blocks, MAX_EXPERTS]
-  float*   dz;            // [max_tokens, pool_size] route_bwd scratch
+  float*   dz;            // route_bwd scratch: fp32 [max_tokens, pool_size], or bf16 [max_tokens, ceil64(pool_size)]
+  int32_t* split_any;     // [4]   which bf16 terms of the split router weights are non-zero
+  void*    w_split;       // [3, pool_size, d] bf16 terms of the router weights (bf16 mode)
   void*    dXp;           // [row_capacity, d] expert_bwd scratch (ctx dtype)
   size_t   bytes;         // total
 };
@@ -164,6 +167,16 @@ struct PoolWgradArgs {
   const void* Xp; const void* A; const void* dYp; const void* dGU;
   int expert_base; int n_experts; float* dW_gu; float* dW_down; bool overwrite;
 };
+int route_tc_launch(unipool_ctx*, const void* x, int T, const float* W_r, float sigma, const float* bias,
+                    int n_experts, int32_t* idx, float* gate, int32_t* counts, float* score_sum,
+                    float* znorm, float* z_saved, cudaStream_t);
+int route_bwd_tc_launch(unipool_ctx*, const void* x, int T, const float* W_r, float sigma, int n_experts,
+                        const float* znorm, const float* z_saved, const int32_t* idx, const float* dgate,
+                        const float* coef, void* dx, float* dW_r, float* dsigma, cudaStream_t);
+int tc_operand_map(unipool_ctx*, void* out_tensor_map, const void* base, uint64_t cols, uint64_t rows,
+                   uint32_t box_rows);
+int router_bwd_gemms_tc(unipool_ctx*, const void* dz16, int Mp, const void* W16, const void* x, int T, int M,
+                        void* dx, float* dW_r, cudaStream_t);
 int expert_fwd_simt(unipool_ctx*, const ExpertFwdArgs&, cudaStream_t);
 int expert_bwd_simt(unipool_ctx*, const ExpertBwdArgs&, cudaStream_t);
 int pool_wgrad_simt(unipool_ctx*, const PoolWgradArgs&, cudaStream_t);

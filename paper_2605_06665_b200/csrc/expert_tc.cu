@@ -50,7 +50,8 @@ struct GemmParams {
   int layer_stride_rows;        // wgrad
   int Mdim, Ndim, Kdim;         // wgrad: dW is [Mdim, Ndim]; row tiles: output columns, contraction
   int f;                        // expert width (fwd1 / dgrad1 addressing)
-  int overwrite;                // wgrad: 1 = dW is written, 0 = dW is added to
+  int overwrite;                // 1 = the output is written, 0 = it is added to (wgrad, dgrad2)
+  int uniform_rows;             // wgrad without offsets: group e = rows [e*Kdim, (e+1)*Kdim) of this many
   int32_t* status;
 };
 
@@ -72,7 +73,7 @@ struct TileCoord { int e, mt, nt, kblocks; bool valid; };
 template <int MODE>
 __device__ __forceinline__ int tiles_total(const GemmParams& p, int& n_nt, int& n_mt) {
   if constexpr (Traits<MODE>::kRowTiles) {
-    n_mt = *p.offsets / BM;
+    n_mt = p.offsets ? *p.offsets / BM : p.Mdim;     // no offsets: one group of Mdim row tiles
     const int ncols = MODE == kFwd1 ? BN / 2 : BN;
     n_nt = (p.Ndim + ncols - 1) / ncols;
     return n_mt * n_nt;
@@ -89,7 +90,7 @@ __device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int tile, i
   if constexpr (Traits<MODE>::kRowTiles) {
     c.mt = tile / n_nt;
     c.nt = tile % n_nt;
-    c.e = p.tile_expert[c.mt];
+    c.e = p.tile_expert ? p.tile_expert[c.mt] : 0;
     c.kblocks = p.Kdim / BK;
     c.valid = c.e >= 0 && c.e < p.n_experts;
   } else {
@@ -99,9 +100,14 @@ __device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int tile, i
     c.mt = rem / n_nt;
     c.nt = rem % n_nt;
     int kb = 0;
-    for (int l = 0; l < p.n_layers; ++l) {
-      const int32_t* off = p.offsets + (int64_t)l * (p.n_experts + 1);
-      kb += (off[c.e + 1] - off[c.e]) / BK;
+    if (p.offsets == nullptr) {
+      const int left = p.uniform_rows - c.e * p.Kdim;
+      kb = (left < p.Kdim ? left : p.Kdim) / BK;
+    } else {
+      for (int l = 0; l < p.n_layers; ++l) {
+        const int32_t* off = p.offsets + (int64_t)l * (p.n_experts + 1);
+        kb += (off[c.e + 1] - off[c.e]) / BK;
+      }
     }
     c.kblocks = kb;
     c.valid = kb > 0;
@@ -215,8 +221,13 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
         const int pe = p.expert_base + c.e;
         int layer = 0, r = 0, r_end = 0;              // wgrad: walks the rows of expert e, layer by layer
         if constexpr (!TR::kRowTiles) {
-          r = p.offsets[c.e];
-          r_end = p.offsets[c.e + 1];
+          if (p.offsets == nullptr) {
+            r = c.e * p.Kdim;
+            r_end = r + c.kblocks * BK;
+          } else {
+            r = p.offsets[c.e];
+            r_end = p.offsets[c.e + 1];
+          }
         }
         for (int kb = 0; kb < c.kblocks; ++kb) {
           if (!tc::mbar_wait(&empty_bar[stage], phase ^ 1u, abort)) { report_timeout(p, abort, 1); ok = false; break; }
@@ -413,7 +424,8 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
           tc::fence_proxy_async();
           __syncwarp();
           if (lane == 0) {
-            tc::tma_store_2d(&tmC0, buf, col, row0);
+            if (MODE == kFwd2 || p.overwrite) tc::tma_store_2d(&tmC0, buf, col, row0);
+            else tc::tma_reduce_add_2d(&tmC0, buf, col, row0);
             tc::bulk_commit();
           }
         }
@@ -459,7 +471,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
       } else {
         const int m0 = row0;                           // row of dW[e]
         if (m0 < p.Mdim) {
-          const int grow = (p.expert_base + c.e) * p.Mdim + m0;
+          const int grow = (p.offsets ? (p.expert_base + c.e) * p.Mdim : 0) + m0;
 #pragma unroll 1
           for (int ch = 0; ch < BN / kChunk; ++ch) {
             const int col = c.nt * BN + ch * kChunk;
@@ -660,7 +672,7 @@ int expert_bwd_tc(unipool_ctx* ctx, const ExpertBwdArgs& a, cudaStream_t s) {
   if ((rc = map_2d(ctx, &tmA, a.dGU, 2 * f, cap, 64, BM)) != UNIPOOL_OK) return rc;
   if ((rc = map_2d(ctx, &tmB, a.W_gu, d, (uint64_t)M * 2 * f, 64, 64)) != UNIPOOL_OK) return rc;
   if ((rc = map_chunk(ctx, &tmC0, a.dXp, d, cap, kMapBf16Chunk)) != UNIPOOL_OK) return rc;
-  p.Ndim = d; p.Kdim = 2 * f;
+  p.Ndim = d; p.Kdim = 2 * f; p.overwrite = 1;
   if ((rc = launch<kDgrad2>(ctx, UNIPOOL_PH_DGRAD_GU, tmA, tmB, tmC0, tmC0, p, s)) != UNIPOOL_OK) return rc;
   if (a.wgrad) {
     PoolWgradArgs w{1, 0, a.offsets, a.Xp, a.A, a.dYp, a.dGU, a.expert_base, a.n_experts, a.dW_gu, a.dW_down,
@@ -671,5 +683,42 @@ int expert_bwd_tc(unipool_ctx* ctx, const ExpertBwdArgs& a, cudaStream_t s) {
 }
 
 int pool_wgrad_tc(unipool_ctx* ctx, const PoolWgradArgs& a, cudaStream_t s) { return wgrad_pair(ctx, a, s); }
+
+int tc_operand_map(unipool_ctx* ctx, void* out, const void* base, uint64_t cols, uint64_t rows, uint32_t box_rows) {
+  return map_2d(ctx, static_cast<CUtensorMap*>(out), base, cols, rows, 64, box_rows);
+}
+
+// Router backward GEMMs (bf16 mode).  dz16 [T, Mp] bf16 (Mp = M rounded up to 64, pad columns
+// zero), W16 [M, d] bf16, x [T, d] bf16:
+//   dx [T, d] bf16 += dz16 W16        (row tiles, one group, TMA add-reduce into dx)
+//   dW_r [M, d] fp32 += dz16^T x      (tokens split evenly over the CTAs, TMA add-reduce)
+int router_bwd_gemms_tc(unipool_ctx* ctx, const void* dz16, int Mp, const void* W16, const void* x, int T, int M,
+                        void* dx, float* dW_r, cudaStream_t s) {
+  const int d = ctx->cfg.d_model;
+  GemmParams p{};
+  p.status = ctx->ws.status;
+  p.n_experts = 1;
+  CUtensorMap tmA, tmB, tmC;
+  int rc;
+  if ((rc = map_2d(ctx, &tmA, dz16, Mp, T, 64, BM)) != UNIPOOL_OK) return rc;
+  if ((rc = map_2d(ctx, &tmB, W16, d, M, 64, 64)) != UNIPOOL_OK) return rc;
+  if ((rc = map_chunk(ctx, &tmC, dx, d, T, kMapBf16Chunk)) != UNIPOOL_OK) return rc;
+  p.Mdim = (T + BM - 1) / BM; p.Ndim = d; p.Kdim = Mp; p.overwrite = 0;
+  if ((rc = launch<kDgrad2>(ctx, UNIPOOL_PH_ROUTE_BWD_DX, tmA, tmB, tmC, tmC, p, s)) != UNIPOOL_OK) return rc;
+
+  const int out_tiles = ((M + BM - 1) / BM) * ((d + BN - 1) / BN);
+  const int t64 = (T + 63) / 64;
+  int splits = ctx->sm_count / out_tiles;
+  if (splits < 1) splits = 1;
+  if (splits > t64) splits = t64;
+  const int chunk = ((t64 + splits - 1) / splits) * 64;
+  splits = (t64 * 64 + chunk - 1) / chunk;
+  if ((rc = map_2d(ctx, &tmA, dz16, Mp, T, 64, 64)) != UNIPOOL_OK) return rc;
+  if ((rc = map_2d(ctx, &tmB, x, d, T, 64, 64)) != UNIPOOL_OK) return rc;
+  if ((rc = map_chunk(ctx, &tmC, dW_r, d, M, kMapF32Chunk)) != UNIPOOL_OK) return rc;
+  p.n_experts = splits; p.n_layers = 1; p.uniform_rows = t64 * 64;
+  p.Mdim = M; p.Ndim = d; p.Kdim = chunk; p.overwrite = 0;
+  return launch<kWgrad>(ctx, UNIPOOL_PH_ROUTE_BWD_DW, tmA, tmB, tmC, tmC, p, s);
+}
 
 }  // namespace unipool

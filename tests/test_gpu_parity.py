@@ -213,6 +213,31 @@ def test_tiny_fp32_end_to_end():
     st.close()
 
 
+def test_fp32_router_weights_in_bf16_mode():
+    """Router weights are fp32 numbers even when activations are bf16: the tensor-core logits
+    (weights split into three bf16 terms) must still be the fp32 logits of the unrounded weights."""
+    import torch
+    cfg = small_cfg(dtype="bf16", d=256, f=128, M=40, k=2, L=1)
+    T = 700
+    inputs = synth.make_inputs(cfg, seed=8, T=T)
+    rng = np.random.default_rng(11)
+    W = (inputs["routers"][0]["W_r"] * (1.0 + 1e-3 * rng.standard_normal((40, 256)))).astype(np.float32)
+    assert (synth.round_to_bf16(W) != W).any()
+    inputs["routers"][0]["W_r"] = W
+    st = build_stack(cfg, inputs, T=T)
+    st.x[0].copy_(torch.from_numpy(inputs["x0"]))
+    st.forward_layer(0)
+    torch.cuda.synchronize()
+    ref = O.route(f64(inputs["x0"]), f64(W), 1.0, st.c, synth.EPS, 2)
+    assert rel_max(to_np(st.z[0]), ref["z"]) < 1e-5
+    check_routing(to_np(st.idx[0]), ref["z"], ref["idx"], 2)
+    ref = O.route(f64(inputs["x0"]), f64(W), 1.0, st.c, synth.EPS, 2, forced_idx=to_np(st.idx[0]))
+    assert rel_max(to_np(st.gate[0]), ref["g"]) < 1e-5
+    assert rel_max(to_np(st.score_sum[0]), ref["S"]) < 1e-5
+    st.ctx.check_status()
+    st.close()
+
+
 def test_empty_batch():
     import torch
     cfg = small_cfg()
