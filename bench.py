@@ -188,6 +188,13 @@ def run_ours(args):
     for _ in range(max(args.warmup, 3)):
         device_step()
     st.ctx.check_status()
+    if args.kernels_only:                    # profiler runs: nothing but the steps themselves
+        timed(device_step, args.steps)
+        st.ctx.check_status()
+        st.close()
+        if rank == 0:
+            print(json.dumps({"kernels_only": True, "workload": args.workload, "steps": args.steps}))
+        return
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
@@ -340,6 +347,8 @@ def main():
                          "backward instead of contracting all layers' rows per expert in one pass at the end")
     ap.add_argument("--cpu-tokens", type=int, default=16384, help="token sample of the CPU-oracle baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--kernels-only", action="store_true",
+                    help="run warm-up and timed steps only and print no result (for runs under a profiler)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

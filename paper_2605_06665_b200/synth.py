@@ -33,6 +33,8 @@ CONFIGS = {
     "978m":           dict(L=24, d=1536, f=4096, M=192, k=2, T=32768, dtype="bf16", private=0, zipf_beta=0.0),
     "978m_pool128":   dict(L=24, d=1536, f=4096, M=128, k=2, T=32768, dtype="bf16", private=0, zipf_beta=0.0),
     "978m_vanilla":   dict(L=24, d=1536, f=4096, M=192, k=2, T=32768, dtype="bf16", private=8, zipf_beta=0.0),
+    # a quarter of one 182m layer (same rows per expert, same tiles): small profiler captures
+    "182m_slice":     dict(L=1,  d=768,  f=2048, M=24,  k=2, T=4096,  dtype="bf16", private=0, zipf_beta=0.0),
     "fine_zipf":      dict(L=12, d=768,  f=512,  M=384, k=8, T=16384, dtype="bf16", private=0, zipf_beta=0.4),
 }
 
