@@ -133,6 +133,30 @@ int unipool_dispatch(unipool_ctx* ctx, const void* x, int32_t T, const int32_t* 
                      int32_t n_experts, int32_t* offsets, int32_t* row_of, int32_t* token_of,
                      int32_t* tile_expert, void* Xp, unipool_stream stream);
 
+/* unipool_dispatch for callers that cannot hand over a workspace (the paper has no counterpart).
+ * Some embedders of this library run where device allocation is off limits: inside a
+ * memory-planned runtime whose arena is fixed before the first step, or in a plugin that only
+ * receives the tensors of one call.  They cannot size and allocate the context's workspace, so
+ * this call needs none and no unipool_ctx: the per-chunk histograms the permutation kernels use as
+ * scratch live in a 2 MiB array inside the library's own device image (each GPU that loads the
+ * library holds it until the process exits).  The call itself never allocates or frees memory.
+ * Same inputs, outputs and results as unipool_dispatch, for d_model/dtype/top_k given here and
+ * row_capacity = rows of the permuted buffers (a multiple of UNIPOOL_ROW_ALIGN, at least
+ * T*top_k + n_experts*(UNIPOOL_ROW_ALIGN-1) rounded up).
+ *   - Limit: ceil(T/64) * n_experts <= 524224 (e.g. 65536 tokens at 511 experts); beyond it the
+ *     call fails with UNIPOOL_ERR_WORKSPACE and launches nothing.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current); make that first call outside any stream capture.
+ *   - All calls share the one array, which keeps the previous call's contents; the kernels
+ *     rewrite every entry they read, so nothing needs clearing.  Two calls that overlap on the
+ *     GPU (different streams) race on it: serialise them.
+ *   - An expert index outside [0, n_experts) is dropped (its row_of entry is -1); without a
+ *     context there is no status word to report it through. */
+int unipool_dispatch_static(const void* x, int32_t T, int32_t d_model, int32_t dtype, int32_t top_k,
+                            const int32_t* idx, int32_t n_experts, int64_t row_capacity,
+                            int32_t* offsets, int32_t* row_of, int32_t* token_of,
+                            int32_t* tile_expert, void* Xp, unipool_stream stream);
+
 /* Grouped SwiGLU expert FFN over the permuted rows (Eq. 2's e_i; App. B):
  *   GU = Xp [W_gate; W_up]^T,  A = silu(G) * U,  Yp = A W_down^T   per group,
  * group e using pool expert expert_base + e.

@@ -23,7 +23,7 @@ EXPORTS = (
     "unipool_last_error", "unipool_check_status", "unipool_route", "unipool_dispatch",
     "unipool_expert_fwd", "unipool_combine", "unipool_expert_bwd", "unipool_pool_wgrad",
     "unipool_pool_aux_loss", "unipool_route_bwd", "unipool_calibrate_c",
-    "unipool_profile_enable", "unipool_profile_read",
+    "unipool_profile_enable", "unipool_profile_read", "unipool_dispatch_static",
 )
 
 PHASES = (
@@ -78,6 +78,8 @@ def lib():
     L.unipool_route.argtypes = [vp, vp, i32, vp, f32, vp, i32, vp, vp, vp, vp, vp, vp, vp]
     L.unipool_dispatch.restype = ctypes.c_int
     L.unipool_dispatch.argtypes = [vp, vp, i32, vp, i32, vp, vp, vp, vp, vp, vp]
+    L.unipool_dispatch_static.restype = ctypes.c_int
+    L.unipool_dispatch_static.argtypes = [vp, i32, i32, i32, i32, vp, i32, i64, vp, vp, vp, vp, vp, vp]
     L.unipool_expert_fwd.restype = ctypes.c_int
     L.unipool_expert_fwd.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp]
     L.unipool_combine.restype = ctypes.c_int
@@ -126,6 +128,15 @@ def row_capacity(cfg):
 
 def workspace_bytes(cfg):
     return int(lib().unipool_workspace_bytes(ctypes.byref(cfg)))
+
+
+def dispatch_static(x, T, d_model, dtype, top_k, idx, n_experts, row_capacity, offsets, row_of, token_of,
+                    tile_expert, Xp):
+    """unipool_dispatch_static: the token permute for callers without a workspace or a context
+    (its scratch is built into the library; it allocates nothing)."""
+    _check(lib().unipool_dispatch_static(_p(x), T, d_model, dtype, top_k, _p(idx), n_experts, row_capacity,
+                                         _p(offsets), _p(row_of), _p(token_of), _p(tile_expert), _p(Xp),
+                                         _stream()))
 
 
 class Context:

@@ -360,3 +360,79 @@ int unpermute_sum_launch(unipool_ctx* ctx, const void* dXp, const int32_t* row_o
 }
 
 }  // namespace unipool
+
+// ---------------------------------------------------------------- dispatch without a workspace
+// Scratch of unipool_dispatch_static: the per-chunk histograms of the map kernels plus a status
+// word, held in the library's own device image.  Every GPU that loads the library carries these
+// 2 MiB until the process exits.  All calls share them.
+namespace {
+constexpr int64_t kStaticHistInts = 1024 * 512 - 64;      // chunks x experts that fit
+static __device__ __align__(256) int32_t g_dispatch_scratch[1024 * 512];
+constexpr int kMaxDevices = 64;
+int32_t* g_scratch_addr[kMaxDevices] = {};
+int g_scratch_sms[kMaxDevices] = {};
+}  // namespace
+
+extern "C" int unipool_dispatch_static(const void* x, int32_t T, int32_t d_model, int32_t dtype, int32_t top_k,
+                                       const int32_t* idx, int32_t n_experts, int64_t row_capacity,
+                                       int32_t* offsets, int32_t* row_of, int32_t* token_of,
+                                       int32_t* tile_expert, void* Xp, unipool_stream stream) {
+  using namespace unipool;
+  UP_REQUIRE(x && idx && offsets && row_of && token_of && tile_expert && Xp, UNIPOOL_ERR_INVALID_ARG,
+             "dispatch_static: a tensor pointer is NULL");
+  UP_REQUIRE(dtype == UNIPOOL_FP32 || dtype == UNIPOOL_BF16, UNIPOOL_ERR_INVALID_ARG, "dispatch_static: bad dtype %d", dtype);
+  const size_t eb = dtype == UNIPOOL_BF16 ? 2 : 4;
+  UP_REQUIRE(d_model > 0 && ((size_t)d_model * eb) % 16 == 0, UNIPOOL_ERR_UNSUPPORTED,
+             "dispatch_static: a row of %d elements is not a whole number of 16-byte vectors", d_model);
+  UP_REQUIRE(n_experts >= 1 && n_experts <= UNIPOOL_MAX_EXPERTS && top_k >= 1 && top_k <= UNIPOOL_MAX_TOPK &&
+                 top_k <= n_experts, UNIPOOL_ERR_UNSUPPORTED, "dispatch_static: bad (n_experts, top_k) = (%d, %d)",
+             n_experts, top_k);
+  UP_REQUIRE(T >= 0 && (int64_t)T * top_k < (1ll << 30), UNIPOOL_ERR_UNSUPPORTED, "dispatch_static: bad T = %d", T);
+  const int64_t need_rows = ((int64_t)T * top_k + (int64_t)n_experts * (UNIPOOL_ROW_ALIGN - 1) + UNIPOOL_ROW_ALIGN - 1) /
+                            UNIPOOL_ROW_ALIGN * UNIPOOL_ROW_ALIGN;
+  UP_REQUIRE(row_capacity % UNIPOOL_ROW_ALIGN == 0 && row_capacity >= need_rows && row_capacity < (1ll << 31),
+             UNIPOOL_ERR_INVALID_ARG, "dispatch_static: row_capacity %lld, need a multiple of %d >= %lld",
+             (long long)row_capacity, UNIPOOL_ROW_ALIGN, (long long)need_rows);
+  const int n_blocks = (T + kDispatchChunkTokens - 1) / kDispatchChunkTokens;
+  UP_REQUIRE((int64_t)n_blocks * n_experts <= kStaticHistInts, UNIPOOL_ERR_WORKSPACE,
+             "dispatch_static: ceil(T/%d) * n_experts = %lld exceeds the built-in scratch of %lld entries "
+             "(use unipool_dispatch with a workspace)", kDispatchChunkTokens, (long long)n_blocks * n_experts,
+             (long long)kStaticHistInts);
+  int dev = 0;
+  UP_CUDA(cudaGetDevice(&dev));
+  UP_REQUIRE(dev >= 0 && dev < kMaxDevices, UNIPOOL_ERR_UNSUPPORTED, "dispatch_static: device ordinal %d", dev);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (g_scratch_addr[dev] == nullptr) {
+    // Once per device, with that device current: in host code the array's name is only a handle,
+    // the kernels need the address it has on THIS device.
+    int32_t* ptr = nullptr;
+    UP_CUDA(cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_dispatch_scratch));
+    int sms = 0;
+    UP_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    g_scratch_sms[dev] = sms;
+    g_scratch_addr[dev] = ptr;
+  }
+  int32_t* status = g_scratch_addr[dev];                   // [0, 64): status word (+ spare)
+  int32_t* bh = g_scratch_addr[dev] + 64;                  // per-chunk histograms / bases
+  const int cap = (int)row_capacity;
+  if (T == 0) {
+    dispatch_empty_kernel<<<(cap + 255) / 256, 256, 0, s>>>(offsets, token_of, tile_expert, n_experts, cap);
+    UP_LAUNCH_CHECK();
+    return UNIPOOL_OK;
+  }
+  // the histograms are fully rewritten by the first kernel for the chunks of this call; nothing
+  // else in the array has to start at zero
+  dispatch_hist_kernel<<<n_blocks, 32, n_experts * sizeof(int), s>>>(idx, T, top_k, n_experts, bh, status);
+  UP_LAUNCH_CHECK();
+  dispatch_scan_kernel<<<1, 512, 0, s>>>(bh, n_blocks, n_experts, cap, offsets, token_of, tile_expert);
+  UP_LAUNCH_CHECK();
+  dispatch_rank_kernel<<<n_blocks, 32, n_experts * sizeof(int), s>>>(idx, T, top_k, n_experts, bh, row_of, token_of);
+  UP_LAUNCH_CHECK();
+  const int row_vecs = (int)((size_t)d_model * eb / 16);
+  int64_t want = ((int64_t)cap + 7) / 8, lim = (int64_t)g_scratch_sms[dev] * 8;
+  const int grid = (int)(want < 1 ? 1 : (want < lim ? want : lim));
+  gather_rows_kernel<<<grid, 256, 0, s>>>(static_cast<const uint4*>(x), token_of, offsets + n_experts,
+                                          static_cast<uint4*>(Xp), row_vecs, cap);
+  UP_LAUNCH_CHECK();
+  return UNIPOOL_OK;
+}
