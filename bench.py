@@ -109,8 +109,7 @@ def algorithmic_bytes(cfg, cap_rows):
         "route_select": T * m * 4 + T * k * 8 + T * 4,
         "dispatch_gather": T * d * b + R * d * b + R * 4,
         "combine": R * d * b + 2 * T * d * b + T * k * 8,
-        "bwd_scale_gather": T * d * b + R * d * b + R * 4,
-        "bwd_dgate": T * d * b + R * d * b + T * k * 8,
+        "bwd_scale_gather": T * d * b + 2 * R * d * b + T * k * 12,     # dy + Yp read, dYp written, dgate
         "unpermute_sum": R * d * b + 2 * T * d * b + T * k * 4,
     }
 

@@ -59,6 +59,12 @@ Workspace carve_workspace(const unipool_config& cfg, void* base) {
     w.dz = reinterpret_cast<float*>(take((size_t)cfg.max_tokens * per_token));
   }
   w.w_split = cfg.dtype == UNIPOOL_BF16 ? take((size_t)3 * cfg.pool_size * cfg.d_model * 2) : nullptr;
+  {
+    const size_t tiles = ((size_t)cfg.max_tokens + 127) / 128;
+    w.part_counts = reinterpret_cast<int32_t*>(take(tiles * cfg.pool_size * sizeof(int32_t)));
+    w.part_sums = reinterpret_cast<float*>(take(tiles * cfg.pool_size * sizeof(float)));
+    w.part_dsigma = reinterpret_cast<float*>(take((((size_t)cfg.max_tokens + 63) / 64) * sizeof(float)));
+  }
   w.dXp = take((size_t)cap * cfg.d_model * eb);
   w.bytes = off;
   return w;

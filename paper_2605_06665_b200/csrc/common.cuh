@@ -55,6 +55,9 @@ struct Workspace {
   float*   dz;            // route_bwd scratch: fp32 [max_tokens, pool_size], or bf16 [max_tokens, ceil64(pool_size)]
   int32_t* split_any;     // [4]   which bf16 terms of the split router weights are non-zero
   void*    w_split;       // [3, pool_size, d] bf16 terms of the router weights (bf16 mode)
+  int32_t* part_counts;   // [ceil(max_tokens/128), pool_size] per-tile routing counts (bf16 mode)
+  float*   part_sums;     // [ceil(max_tokens/128), pool_size] per-tile score sums
+  float*   part_dsigma;   // [ceil(max_tokens/64)] per-block dsigma terms
   void*    dXp;           // [row_capacity, d] expert_bwd scratch (ctx dtype)
   size_t   bytes;         // total
 };

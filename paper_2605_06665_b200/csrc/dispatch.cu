@@ -28,46 +28,62 @@ dispatch_hist_kernel(const int32_t* __restrict__ idx, int T, int k, int M, int32
   for (int i = lane; i < M; i += 32) block_hist[(int64_t)blockIdx.x * M + i] = hist[i];
 }
 
-// One block: per-expert totals -> padded exclusive scan -> per-(block, expert) bases.
-// block_hist[b][e] is replaced by the first row of block b's assignments to e.
-__global__ void __launch_bounds__(512)
+// One block of 1024 threads: per-expert totals -> padded exclusive scan -> per-(chunk, expert) bases.
+// block_hist[b][e] is replaced by the first row of chunk b's assignments to e.  Thread (seg, e)
+// walks a contiguous segment of chunks for expert e, so that the loads of one pass are independent
+// and coalesced over e.
+constexpr int kScanThreads = 1024;
+__global__ void __launch_bounds__(kScanThreads)
 dispatch_scan_kernel(int32_t* __restrict__ block_hist, int n_blocks, int M, int row_capacity,
                      int32_t* __restrict__ offsets, int32_t* __restrict__ token_of,
                      int32_t* __restrict__ tile_expert) {
-  __shared__ int padded[UNIPOOL_MAX_EXPERTS];
+  __shared__ int part[kScanThreads];                  // [segs][M] chunk-segment sums, then bases
   __shared__ int start[UNIPOOL_MAX_EXPERTS + 1];
   __shared__ int total_s[UNIPOOL_MAX_EXPERTS];
-  const int e = threadIdx.x;
-  int total = 0;
-  if (e < M) {
-    for (int b = 0; b < n_blocks; ++b) total += block_hist[(int64_t)b * M + e];
-    total_s[e] = total;
-    padded[e] = (total + UNIPOOL_ROW_ALIGN - 1) / UNIPOOL_ROW_ALIGN * UNIPOOL_ROW_ALIGN;
+  const int segs = kScanThreads / M < 1 ? 1 : (kScanThreads / M > 32 ? 32 : kScanThreads / M);
+  const int per_seg = (n_blocks + segs - 1) / segs;
+  const int e = threadIdx.x % M, seg = threadIdx.x / M;
+  const bool worker = seg < segs;
+  const int b0 = seg * per_seg, b1 = min(n_blocks, b0 + per_seg);
+  if (worker) {
+    int sum = 0;
+#pragma unroll 8
+    for (int b = b0; b < b1; ++b) sum += block_hist[(int64_t)b * M + e];
+    part[seg * M + e] = sum;
+  }
+  __syncthreads();
+  if (threadIdx.x < M) {                               // totals and segment bases of expert threadIdx.x
+    int run = 0;
+    for (int sg = 0; sg < segs; ++sg) { const int v = part[sg * M + threadIdx.x]; part[sg * M + threadIdx.x] = run; run += v; }
+    total_s[threadIdx.x] = run;
   }
   __syncthreads();
   if (threadIdx.x == 0) {
     int run = 0;
-    for (int i = 0; i < M; ++i) { start[i] = run; run += padded[i]; }
+    for (int i = 0; i < M; ++i) {
+      start[i] = run;
+      run += (total_s[i] + UNIPOOL_ROW_ALIGN - 1) / UNIPOOL_ROW_ALIGN * UNIPOOL_ROW_ALIGN;
+    }
     start[M] = run;
   }
   __syncthreads();
-  if (e < M) offsets[e] = start[e];
-  if (e == 0) offsets[M] = start[M];
-  if (e < M) {
-    int run = start[e];
-    for (int b = 0; b < n_blocks; ++b) {
-      int h = block_hist[(int64_t)b * M + e];
+  if (threadIdx.x <= M) offsets[threadIdx.x] = start[threadIdx.x];
+  if (worker) {
+    int run = start[e] + part[seg * M + e];
+#pragma unroll 8
+    for (int b = b0; b < b1; ++b) {
+      const int h = block_hist[(int64_t)b * M + e];
       block_hist[(int64_t)b * M + e] = run;
       run += h;
     }
   }
   // pad rows of every group, rows beyond the last group, tile -> expert table
   const int used = start[M];
-  for (int g = 0; g < M; ++g) {
-    int lo = start[g] + total_s[g], hi = start[g + 1];
-    for (int r = lo + threadIdx.x; r < hi; r += blockDim.x) token_of[r] = -1;
-    for (int tl = start[g] / UNIPOOL_ROW_ALIGN + threadIdx.x; tl < start[g + 1] / UNIPOOL_ROW_ALIGN; tl += blockDim.x)
-      tile_expert[tl] = g;
+  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+  for (int g = warp; g < M; g += kScanThreads / 32) {
+    const int lo = start[g] + total_s[g], hi = start[g + 1];
+    for (int r = lo + lane; r < hi; r += 32) token_of[r] = -1;
+    for (int tl = start[g] / UNIPOOL_ROW_ALIGN + lane; tl < hi / UNIPOOL_ROW_ALIGN; tl += 32) tile_expert[tl] = g;
   }
   for (int r = used + threadIdx.x; r < row_capacity; r += blockDim.x) token_of[r] = -1;
   for (int tl = used / UNIPOOL_ROW_ALIGN + threadIdx.x; tl < row_capacity / UNIPOOL_ROW_ALIGN; tl += blockDim.x)
@@ -103,11 +119,11 @@ dispatch_rank_kernel(const int32_t* __restrict__ idx, int T, int k, int M,
 }
 
 // ---------------------------------------------------------------- row movers
-// Vector type: 16 bytes.
-template <typename T>
-__device__ __forceinline__ void zero16(uint4& v) { v = make_uint4(0, 0, 0, 0); }
+// One warp moves one row in 16-byte vectors; a lane owns vectors lane, lane + 32, ... and issues
+// all loads of a pass (kVpl vectors per lane and source row) before it uses any of them.
+constexpr int kVpl = 3;
 
-// Xp[r] = x[token_of[r]]  (zero on pad rows), one warp per row, rows < offsets[M].
+// Xp[r] = x[token_of[r]]  (zero on pad rows), rows < offsets[M].
 __global__ void __launch_bounds__(256)
 gather_rows_kernel(const uint4* __restrict__ x, const int32_t* __restrict__ token_of,
                    const int32_t* __restrict__ offsets_end, uint4* __restrict__ Xp, int row_vecs,
@@ -117,11 +133,19 @@ gather_rows_kernel(const uint4* __restrict__ x, const int32_t* __restrict__ toke
   for (int r = blockIdx.x * 8 + warp; r < used; r += gridDim.x * 8) {
     const int t = token_of[r];
     uint4* dst = Xp + (int64_t)r * row_vecs;
-    if (t >= 0) {
-      const uint4* src = x + (int64_t)t * row_vecs;
-      for (int v = lane; v < row_vecs; v += 32) dst[v] = __ldg(src + v);
-    } else {
-      for (int v = lane; v < row_vecs; v += 32) dst[v] = make_uint4(0, 0, 0, 0);
+    const uint4* src = x + (int64_t)(t >= 0 ? t : 0) * row_vecs;
+    for (int v0 = lane; v0 < row_vecs; v0 += 32 * kVpl) {
+      uint4 buf[kVpl];
+#pragma unroll
+      for (int i = 0; i < kVpl; ++i) {
+        const int v = v0 + 32 * i;
+        buf[i] = (t >= 0 && v < row_vecs) ? __ldg(src + v) : make_uint4(0, 0, 0, 0);
+      }
+#pragma unroll
+      for (int i = 0; i < kVpl; ++i) {
+        const int v = v0 + 32 * i;
+        if (v < row_vecs) dst[v] = buf[i];
+      }
     }
   }
 }
@@ -159,7 +183,8 @@ template <> struct Vec16<__nv_bfloat16> {
 };
 
 // y[t] = (residual[t]) + sum_j gate[t,j] * Yp[row_of[t,j]]   (gate == NULL: unit weights)
-template <typename T>
+// KT = compile-time bound of k (registers for the rows in flight).
+template <typename T, int KT>
 __global__ void __launch_bounds__(256)
 combine_kernel(const uint4* __restrict__ Yp, const int32_t* __restrict__ row_of,
                const float* __restrict__ gate, const uint4* __restrict__ residual,
@@ -167,95 +192,112 @@ combine_kernel(const uint4* __restrict__ Yp, const int32_t* __restrict__ row_of,
   constexpr int N = Vec16<T>::N;
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
   for (int t = blockIdx.x * 8 + warp; t < n_tokens; t += gridDim.x * 8) {
-    int rows[UNIPOOL_MAX_TOPK];
-    float g[UNIPOOL_MAX_TOPK];
-    for (int j = 0; j < k; ++j) {
-      rows[j] = row_of[(int64_t)t * k + j];
-      g[j] = gate ? gate[(int64_t)t * k + j] : 1.f;
+    int rows[KT];
+    float g[KT];
+#pragma unroll
+    for (int j = 0; j < KT; ++j) {
+      rows[j] = j < k ? row_of[(int64_t)t * k + j] : -1;
+      g[j] = (j < k && gate) ? gate[(int64_t)t * k + j] : 1.f;
     }
-    for (int v = lane; v < row_vecs; v += 32) {
-      float acc[N];
-      if (residual) {
-        Vec16<T>::unpack(__ldg(residual + (int64_t)t * row_vecs + v), acc);
-      } else {
+    for (int v0 = lane; v0 < row_vecs; v0 += 32 * kVpl) {
+      uint4 rv[kVpl], yv[KT][kVpl];
 #pragma unroll
-        for (int i = 0; i < N; ++i) acc[i] = 0.f;
-      }
-      for (int j = 0; j < k; ++j) {
-        if (rows[j] < 0) continue;
-        float f[N];
-        Vec16<T>::unpack(__ldg(Yp + (int64_t)rows[j] * row_vecs + v), f);
+      for (int i = 0; i < kVpl; ++i) {
+        const int v = v0 + 32 * i;
+        rv[i] = (residual && v < row_vecs) ? __ldg(residual + (int64_t)t * row_vecs + v) : make_uint4(0, 0, 0, 0);
 #pragma unroll
-        for (int i = 0; i < N; ++i) acc[i] = fmaf(g[j], f[i], acc[i]);
+        for (int j = 0; j < KT; ++j)
+          yv[j][i] = (rows[j] >= 0 && v < row_vecs) ? __ldg(Yp + (int64_t)rows[j] * row_vecs + v)
+                                                    : make_uint4(0, 0, 0, 0);
       }
-      y[(int64_t)t * row_vecs + v] = Vec16<T>::pack(acc);
+#pragma unroll
+      for (int i = 0; i < kVpl; ++i) {
+        const int v = v0 + 32 * i;
+        if (v >= row_vecs) continue;
+        float acc[N];
+        if (residual) {
+          Vec16<T>::unpack(rv[i], acc);
+        } else {
+#pragma unroll
+          for (int q = 0; q < N; ++q) acc[q] = 0.f;
+        }
+#pragma unroll
+        for (int j = 0; j < KT; ++j) {
+          if (rows[j] < 0) continue;
+          float fv[N];
+          Vec16<T>::unpack(yv[j][i], fv);
+#pragma unroll
+          for (int q = 0; q < N; ++q) acc[q] = fmaf(g[j], fv[q], acc[q]);
+        }
+        y[(int64_t)t * row_vecs + v] = Vec16<T>::pack(acc);
+      }
     }
   }
 }
 
-// dYp[r] = gate(r) * dy[token_of[r]] (zero on pad rows) for rows < offsets[M];
-// the gate of a row is found through row_of: slot j of token t with row_of[t,j] == r.
-template <typename T>
+// Backward of the combine, token-major: for token t and slot j with row r = row_of[t,j]
+//   dgate[t,j] = <dy[t], Yp[r]>,   dYp[r] = gate[t,j] * dy[t];
+// afterwards the pad rows (token_of < 0) below offsets[M] are zeroed.
+template <typename T, int KT>
 __global__ void __launch_bounds__(256)
-scale_gather_kernel(const uint4* __restrict__ dy, const int32_t* __restrict__ token_of,
-                    const int32_t* __restrict__ row_of, const float* __restrict__ gate,
-                    const int32_t* __restrict__ offsets_end, uint4* __restrict__ dYp, int k,
-                    int row_vecs) {
-  constexpr int N = Vec16<T>::N;
-  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-  const int used = *offsets_end;
-  for (int r = blockIdx.x * 8 + warp; r < used; r += gridDim.x * 8) {
-    const int t = token_of[r];
-    uint4* dst = dYp + (int64_t)r * row_vecs;
-    if (t < 0) {
-      for (int v = lane; v < row_vecs; v += 32) dst[v] = make_uint4(0, 0, 0, 0);
-      continue;
-    }
-    float g = 0.f;
-    for (int j = 0; j < k; ++j)
-      if (row_of[(int64_t)t * k + j] == r) g = gate[(int64_t)t * k + j];
-    const uint4* src = dy + (int64_t)t * row_vecs;
-    for (int v = lane; v < row_vecs; v += 32) {
-      float f[N];
-      Vec16<T>::unpack(__ldg(src + v), f);
-#pragma unroll
-      for (int i = 0; i < N; ++i) f[i] *= g;
-      dst[v] = Vec16<T>::pack(f);
-    }
-  }
-}
-
-// dgate[t,j] = <dy[t], Yp[row_of[t,j]]>, one warp per token.
-template <typename T>
-__global__ void __launch_bounds__(256)
-dgate_kernel(const uint4* __restrict__ dy, const uint4* __restrict__ Yp,
-             const int32_t* __restrict__ row_of, float* __restrict__ dgate, int n_tokens, int k,
-             int row_vecs) {
+combine_bwd_kernel(const uint4* __restrict__ dy, const uint4* __restrict__ Yp,
+                   const int32_t* __restrict__ row_of, const float* __restrict__ gate,
+                   const int32_t* __restrict__ token_of, const int32_t* __restrict__ offsets_end,
+                   uint4* __restrict__ dYp, float* __restrict__ dgate, int n_tokens, int k, int row_vecs) {
   constexpr int N = Vec16<T>::N;
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
   for (int t = blockIdx.x * 8 + warp; t < n_tokens; t += gridDim.x * 8) {
-    float acc[UNIPOOL_MAX_TOPK];
-    int rows[UNIPOOL_MAX_TOPK];
+    int rows[KT];
+    float g[KT], dot[KT];
 #pragma unroll
-    for (int j = 0; j < UNIPOOL_MAX_TOPK; ++j) { acc[j] = 0.f; rows[j] = j < k ? row_of[(int64_t)t * k + j] : -1; }
-    for (int v = lane; v < row_vecs; v += 32) {
-      float a[N];
-      Vec16<T>::unpack(__ldg(dy + (int64_t)t * row_vecs + v), a);
+    for (int j = 0; j < KT; ++j) {
+      rows[j] = j < k ? row_of[(int64_t)t * k + j] : -1;
+      g[j] = j < k ? gate[(int64_t)t * k + j] : 0.f;
+      dot[j] = 0.f;
+    }
+    for (int v0 = lane; v0 < row_vecs; v0 += 32 * kVpl) {
+      uint4 dv[kVpl], yv[KT][kVpl];
 #pragma unroll
-      for (int j = 0; j < UNIPOOL_MAX_TOPK; ++j) {
-        if (rows[j] < 0) continue;
-        float f[N];
-        Vec16<T>::unpack(__ldg(Yp + (int64_t)rows[j] * row_vecs + v), f);
+      for (int i = 0; i < kVpl; ++i) {
+        const int v = v0 + 32 * i;
+        dv[i] = v < row_vecs ? __ldg(dy + (int64_t)t * row_vecs + v) : make_uint4(0, 0, 0, 0);
 #pragma unroll
-        for (int i = 0; i < N; ++i) acc[j] = fmaf(a[i], f[i], acc[j]);
+        for (int j = 0; j < KT; ++j)
+          yv[j][i] = (rows[j] >= 0 && v < row_vecs) ? __ldg(Yp + (int64_t)rows[j] * row_vecs + v)
+                                                    : make_uint4(0, 0, 0, 0);
+      }
+#pragma unroll
+      for (int i = 0; i < kVpl; ++i) {
+        const int v = v0 + 32 * i;
+        if (v >= row_vecs) continue;
+        float a[N];
+        Vec16<T>::unpack(dv[i], a);
+#pragma unroll
+        for (int j = 0; j < KT; ++j) {
+          if (rows[j] < 0) continue;
+          float fv[N], o[N];
+          Vec16<T>::unpack(yv[j][i], fv);
+#pragma unroll
+          for (int q = 0; q < N; ++q) {
+            dot[j] = fmaf(a[q], fv[q], dot[j]);
+            o[q] = g[j] * a[q];
+          }
+          dYp[(int64_t)rows[j] * row_vecs + v] = Vec16<T>::pack(o);
+        }
       }
     }
 #pragma unroll
-    for (int j = 0; j < UNIPOOL_MAX_TOPK; ++j) {
+    for (int j = 0; j < KT; ++j) {
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], o);
-      if (lane == 0 && j < k) dgate[(int64_t)t * k + j] = acc[j];
+      for (int o = 16; o > 0; o >>= 1) dot[j] += __shfl_xor_sync(0xffffffffu, dot[j], o);
+      if (lane == 0 && j < k) dgate[(int64_t)t * k + j] = dot[j];
     }
+  }
+  const int used = *offsets_end;
+  for (int r = blockIdx.x * 8 + warp; r < used; r += gridDim.x * 8) {
+    if (token_of[r] >= 0) continue;
+    uint4* dst = dYp + (int64_t)r * row_vecs;
+    for (int v = lane; v < row_vecs; v += 32) dst[v] = make_uint4(0, 0, 0, 0);
   }
 }
 
@@ -289,7 +331,7 @@ int dispatch_launch(unipool_ctx* ctx, const void* x, int T, const int32_t* idx, 
   PhaseTimer pt(ctx, UNIPOOL_PH_DISPATCH_MAPS, 3, s);
   dispatch_hist_kernel<<<n_blocks, 32, M * sizeof(int), s>>>(idx, T, k, M, bh, ctx->ws.status);
   UP_LAUNCH_CHECK();
-  dispatch_scan_kernel<<<1, 512, 0, s>>>(bh, n_blocks, M, cap, offsets, token_of, tile_expert);
+  dispatch_scan_kernel<<<1, kScanThreads, 0, s>>>(bh, n_blocks, M, cap, offsets, token_of, tile_expert);
   UP_LAUNCH_CHECK();
   dispatch_rank_kernel<<<n_blocks, 32, M * sizeof(int), s>>>(idx, T, k, M, bh, row_of, token_of);
   UP_LAUNCH_CHECK();
@@ -302,6 +344,18 @@ int dispatch_launch(unipool_ctx* ctx, const void* x, int T, const int32_t* idx, 
   return UNIPOOL_OK;
 }
 
+template <typename T>
+static void combine_dispatch_k(int grid, cudaStream_t s, int k, const void* Yp, const int32_t* row_of,
+                               const float* gate, const void* residual, void* y, int n_tokens, int row_vecs) {
+  auto Y = static_cast<const uint4*>(Yp);
+  auto R = static_cast<const uint4*>(residual);
+  auto O = static_cast<uint4*>(y);
+  if (k <= 1) combine_kernel<T, 1><<<grid, 256, 0, s>>>(Y, row_of, gate, R, O, n_tokens, k, row_vecs);
+  else if (k <= 2) combine_kernel<T, 2><<<grid, 256, 0, s>>>(Y, row_of, gate, R, O, n_tokens, k, row_vecs);
+  else if (k <= 4) combine_kernel<T, 4><<<grid, 256, 0, s>>>(Y, row_of, gate, R, O, n_tokens, k, row_vecs);
+  else combine_kernel<T, 8><<<grid, 256, 0, s>>>(Y, row_of, gate, R, O, n_tokens, k, row_vecs);
+}
+
 static int combine_phase(unipool_ctx* ctx, int phase, const void* Yp, const int32_t* row_of,
                          const float* gate, int T, const void* residual, void* y, cudaStream_t s) {
   if (T == 0) return UNIPOOL_OK;
@@ -310,11 +364,9 @@ static int combine_phase(unipool_ctx* ctx, int phase, const void* Yp, const int3
   const int row_vecs = (int)((size_t)ctx->cfg.d_model * ctx->elem_bytes / 16);
   const int grid = row_mover_grid(ctx, T);
   if (ctx->cfg.dtype == UNIPOOL_BF16)
-    combine_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>(static_cast<const uint4*>(Yp), row_of, gate,
-        static_cast<const uint4*>(residual), static_cast<uint4*>(y), T, k, row_vecs);
+    combine_dispatch_k<__nv_bfloat16>(grid, s, k, Yp, row_of, gate, residual, y, T, row_vecs);
   else
-    combine_kernel<float><<<grid, 256, 0, s>>>(static_cast<const uint4*>(Yp), row_of, gate,
-        static_cast<const uint4*>(residual), static_cast<uint4*>(y), T, k, row_vecs);
+    combine_dispatch_k<float>(grid, s, k, Yp, row_of, gate, residual, y, T, row_vecs);
   UP_LAUNCH_CHECK();
   return UNIPOOL_OK;
 }
@@ -324,31 +376,31 @@ int combine_launch(unipool_ctx* ctx, const void* Yp, const int32_t* row_of, cons
   return combine_phase(ctx, UNIPOOL_PH_COMBINE, Yp, row_of, gate, T, residual, y, s);
 }
 
+template <typename T>
+static void combine_bwd_dispatch_k(int grid, cudaStream_t s, int k, const void* dy, const void* Yp,
+                                   const int32_t* row_of, const float* gate, const int32_t* token_of,
+                                   const int32_t* offsets_end, void* dYp, float* dgate, int n_tokens, int row_vecs) {
+  auto D = static_cast<const uint4*>(dy);
+  auto Y = static_cast<const uint4*>(Yp);
+  auto O = static_cast<uint4*>(dYp);
+  if (k <= 1) combine_bwd_kernel<T, 1><<<grid, 256, 0, s>>>(D, Y, row_of, gate, token_of, offsets_end, O, dgate, n_tokens, k, row_vecs);
+  else if (k <= 2) combine_bwd_kernel<T, 2><<<grid, 256, 0, s>>>(D, Y, row_of, gate, token_of, offsets_end, O, dgate, n_tokens, k, row_vecs);
+  else if (k <= 4) combine_bwd_kernel<T, 4><<<grid, 256, 0, s>>>(D, Y, row_of, gate, token_of, offsets_end, O, dgate, n_tokens, k, row_vecs);
+  else combine_bwd_kernel<T, 8><<<grid, 256, 0, s>>>(D, Y, row_of, gate, token_of, offsets_end, O, dgate, n_tokens, k, row_vecs);
+}
+
 int combine_bwd_launch(unipool_ctx* ctx, const void* dy, int T, const int32_t* row_of,
                        const float* gate, const int32_t* token_of, const int32_t* offsets, int M,
                        const void* Yp, void* dYp, float* dgate, cudaStream_t s) {
   if (T == 0) return UNIPOOL_OK;
   const int k = ctx->cfg.top_k;
   const int row_vecs = (int)((size_t)ctx->cfg.d_model * ctx->elem_bytes / 16);
-  const int g1 = row_mover_grid(ctx, ctx->row_capacity), g2 = row_mover_grid(ctx, T);
-  const bool bf16 = ctx->cfg.dtype == UNIPOOL_BF16;
-  {
-    PhaseTimer pt(ctx, UNIPOOL_PH_BWD_SCALE_GATHER, 1, s);
-    if (bf16)
-      scale_gather_kernel<__nv_bfloat16><<<g1, 256, 0, s>>>(static_cast<const uint4*>(dy), token_of, row_of,
-          gate, offsets + M, static_cast<uint4*>(dYp), k, row_vecs);
-    else
-      scale_gather_kernel<float><<<g1, 256, 0, s>>>(static_cast<const uint4*>(dy), token_of, row_of, gate,
-          offsets + M, static_cast<uint4*>(dYp), k, row_vecs);
-    UP_LAUNCH_CHECK();
-  }
-  PhaseTimer pt(ctx, UNIPOOL_PH_BWD_DGATE, 1, s);
-  if (bf16)
-    dgate_kernel<__nv_bfloat16><<<g2, 256, 0, s>>>(static_cast<const uint4*>(dy), static_cast<const uint4*>(Yp),
-        row_of, dgate, T, k, row_vecs);
+  const int grid = row_mover_grid(ctx, T);
+  PhaseTimer pt(ctx, UNIPOOL_PH_BWD_SCALE_GATHER, 1, s);
+  if (ctx->cfg.dtype == UNIPOOL_BF16)
+    combine_bwd_dispatch_k<__nv_bfloat16>(grid, s, k, dy, Yp, row_of, gate, token_of, offsets + M, dYp, dgate, T, row_vecs);
   else
-    dgate_kernel<float><<<g2, 256, 0, s>>>(static_cast<const uint4*>(dy), static_cast<const uint4*>(Yp),
-        row_of, dgate, T, k, row_vecs);
+    combine_bwd_dispatch_k<float>(grid, s, k, dy, Yp, row_of, gate, token_of, offsets + M, dYp, dgate, T, row_vecs);
   UP_LAUNCH_CHECK();
   return UNIPOOL_OK;
 }
@@ -424,7 +476,7 @@ extern "C" int unipool_dispatch_static(const void* x, int32_t T, int32_t d_model
   // else in the array has to start at zero
   dispatch_hist_kernel<<<n_blocks, 32, n_experts * sizeof(int), s>>>(idx, T, top_k, n_experts, bh, status);
   UP_LAUNCH_CHECK();
-  dispatch_scan_kernel<<<1, 512, 0, s>>>(bh, n_blocks, n_experts, cap, offsets, token_of, tile_expert);
+  dispatch_scan_kernel<<<1, kScanThreads, 0, s>>>(bh, n_blocks, n_experts, cap, offsets, token_of, tile_expert);
   UP_LAUNCH_CHECK();
   dispatch_rank_kernel<<<n_blocks, 32, n_experts * sizeof(int), s>>>(idx, T, top_k, n_experts, bh, row_of, token_of);
   UP_LAUNCH_CHECK();

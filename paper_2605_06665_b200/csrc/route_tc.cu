@@ -29,7 +29,7 @@ struct RouteParams {
   float sigma_c, eps;
   int32_t* idx; float* gate; float* znorm; float* z_saved;
   int32_t* counts_out; float* sum_out;
-  int32_t* acc_counts; double* acc_sums; uint32_t* ticket;
+  int32_t* part_counts; float* part_sums; uint32_t* ticket;   // per-tile statistics [tiles][M]
   const int32_t* split_any;            // [3] does split s hold a non-zero anywhere
   int stages;                          // operand stages that fit into shared memory
   uint32_t w_bytes;                    // bytes of one W k-block: ceil(M / 128) boxes of 128 rows
@@ -273,21 +273,25 @@ route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     // the four epilogue warps publish the tile's statistics (named barrier 1: 128 threads)
     asm volatile("bar.sync 1, 128;" ::: "memory");
     for (int i = threadIdx.x; i < M; i += kTile) {
-      const float s = (wsum[i] + wsum[M + i]) + (wsum[2 * M + i] + wsum[3 * M + i]);
-      if (hist[i]) atomicAdd(&p.acc_counts[i], hist[i]);
-      if (s != 0.f) atomicAdd(&p.acc_sums[i], (double)s);
+      p.part_counts[(int64_t)blockIdx.x * M + i] = hist[i];
+      p.part_sums[(int64_t)blockIdx.x * M + i] = (wsum[i] + wsum[M + i]) + (wsum[2 * M + i] + wsum[3 * M + i]);
     }
     __threadfence();
     asm volatile("bar.sync 1, 128;" ::: "memory");
     if (threadIdx.x == 0) *last_flag = atomicAdd(p.ticket, 1u) == gridDim.x - 1 ? 1 : 0;
     asm volatile("bar.sync 1, 128;" ::: "memory");
-    if (*last_flag) {                     // the block that arrives last publishes and resets
+    if (*last_flag) {                     // the CTA that arrives last adds the tiles up, in tile order
       __threadfence();
       for (int i = threadIdx.x; i < M; i += kTile) {
-        p.counts_out[i] = __ldcg(&p.acc_counts[i]);
-        p.sum_out[i] = (float)__ldcg(&p.acc_sums[i]);
-        p.acc_counts[i] = 0;
-        p.acc_sums[i] = 0.0;
+        int cnt = 0;
+        double sum = 0.0;
+#pragma unroll 8
+        for (int b = 0; b < (int)gridDim.x; ++b) {
+          cnt += __ldcg(&p.part_counts[(int64_t)b * M + i]);
+          sum += (double)__ldcg(&p.part_sums[(int64_t)b * M + i]);
+        }
+        p.counts_out[i] = cnt;
+        p.sum_out[i] = (float)sum;
       }
       if (threadIdx.x == 0) *p.ticket = 0u;
     }
@@ -386,7 +390,7 @@ int route_tc_launch(unipool_ctx* ctx, const void* x, int T, const float* W_r, fl
   p.sigma_c = sigma * ctx->cfg.c; p.eps = ctx->cfg.eps;
   p.idx = idx; p.gate = gate; p.znorm = znorm; p.z_saved = z_saved;
   p.counts_out = counts; p.sum_out = score_sum;
-  p.acc_counts = ctx->ws.route_counts; p.acc_sums = ctx->ws.route_sums; p.ticket = ctx->ws.tickets + 0;
+  p.part_counts = ctx->ws.part_counts; p.part_sums = ctx->ws.part_sums; p.ticket = ctx->ws.tickets + 0;
   p.split_any = ctx->ws.split_any;
   p.status = ctx->ws.status;
   p.w_bytes = (uint32_t)((M + 127) / 128) * 16384u;
