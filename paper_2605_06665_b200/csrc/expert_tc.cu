@@ -22,7 +22,8 @@ namespace {
 constexpr int BM = 128;          // rows of an output tile (TMEM lanes)
 constexpr int BN = 256;          // columns of an output tile (one tcgen05.mma of N = 256)
 constexpr int BK = 64;           // k-block: 64 bf16 = one 128-byte swizzle row
-constexpr int kThreads = 192;
+constexpr int kThreads = 192;           // producer warp, MMA warp, four epilogue warps
+constexpr int kThreadsIo = 320;         // dgrad1: plus four warps that move the epilogue's operands
 constexpr int kEpiWarps = 4;
 constexpr uint32_t kABytes = BM * BK * 2;
 constexpr uint32_t kBBytes = BN * BK * 2;
@@ -59,6 +60,7 @@ struct GemmParams {
 // The SwiGLU-derivative epilogue also reads G and U, so it trades one operand stage
 // for a ring of five (G, U) chunk buffers per warp that are fetched three chunks ahead.
 template <int MODE> struct Traits {
+  static constexpr int kThreads = MODE == 2 ? kThreadsIo : unipool::kThreads;
   static constexpr int kStages = MODE == 2 ? 3 : 4;
   static constexpr uint32_t kStagingOffset = kStages * kStageBytes;
   static constexpr uint32_t kStagingPerWarp = MODE == 2 ? 20480 : 8192;
@@ -165,8 +167,37 @@ __device__ __forceinline__ void unstage_row_bf16(uint8_t* tile, int r, float (&v
   }
 }
 
+// dgrad1: the (G, U) chunks of one epilogue warp's rows, over all tiles of this CTA, in the
+// order the epilogue consumes them.  Chunk number n of the stream uses ring slot n % kRing.
+constexpr int kRing = 5, kAhead = 3;                   // ring slots per warp, prefetch distance
 template <int MODE>
-__global__ void __launch_bounds__(kThreads, 1)
+struct ChunkCursor {
+  int tile, ch, nch, nt, row0;
+  __device__ void seek(const GemmParams& p, int total, int n_nt, int n_mt, int quarter) {
+    while (tile < total) {                              // next tile that has chunks
+      const TileCoord c = tile_coord<MODE>(p, tile, n_nt, n_mt);
+      if (c.valid) {
+        nt = c.nt;
+        row0 = c.mt * BM + quarter * 32;
+        nch = min(BN / kChunk, (p.f - c.nt * BN) / kChunk);
+        ch = 0;
+        if (nch > 0) return;
+      }
+      tile += gridDim.x;
+    }
+  }
+  __device__ void start(const GemmParams& p, int total, int n_nt, int n_mt, int quarter) {
+    tile = blockIdx.x; ch = 0; nch = 0; nt = 0; row0 = 0;
+    seek(p, total, n_nt, n_mt, quarter);
+  }
+  __device__ void next(const GemmParams& p, int total, int n_nt, int n_mt, int quarter) {
+    if (++ch == nch) { tile += gridDim.x; seek(p, total, n_nt, n_mt, quarter); }
+  }
+  __device__ int col() const { return nt * BN + ch * kChunk; }
+};
+
+template <int MODE>
+__global__ void __launch_bounds__(Traits<MODE>::kThreads, 1)
 grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                        const __grid_constant__ CUtensorMap tmC0, const __grid_constant__ CUtensorMap tmC1,
                        const GemmParams p) {
@@ -180,8 +211,9 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
   uint64_t* empty_bar = full_bar + kStages;
   uint64_t* tmem_full = empty_bar + kStages;
   uint64_t* tmem_empty = tmem_full + 2;
-  uint64_t* epi_bar = tmem_empty + 2;               // [kEpiWarps][5] operand loads of the epilogue
-  uint32_t* tmem_ptr = reinterpret_cast<uint32_t*>(epi_bar + 5 * kEpiWarps);
+  uint64_t* epi_bar = tmem_empty + 2;               // [kEpiWarps][5] operand loads of the epilogue have landed
+  uint64_t* staged_bar = epi_bar + 5 * kEpiWarps;   // [kEpiWarps][5] results are staged, ready to store
+  uint32_t* tmem_ptr = reinterpret_cast<uint32_t*>(staged_bar + 5 * kEpiWarps);
   volatile int* abort = reinterpret_cast<volatile int*>(tmem_ptr + 1);
 
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
@@ -189,7 +221,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { tc::mbar_init(&full_bar[s], 1); tc::mbar_init(&empty_bar[s], 1); }
     for (int a = 0; a < 2; ++a) { tc::mbar_init(&tmem_full[a], 1); tc::mbar_init(&tmem_empty[a], kEpiWarps); }
-    for (int i = 0; i < 5 * kEpiWarps; ++i) tc::mbar_init(&epi_bar[i], 1);
+    for (int i = 0; i < 5 * kEpiWarps; ++i) { tc::mbar_init(&epi_bar[i], 1); tc::mbar_init(&staged_bar[i], 1); }
     *abort = 0;
     tc::fence_barrier_init();
     tc::tma_prefetch_desc(&tmA);
@@ -305,6 +337,51 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
         if (ok) tc::umma_commit(&tmem_full[acc]);        // accumulator complete
       }
     }
+  } else if (warp >= 6) {
+    // ------------------------------------------------------------ dgrad1: operand mover of epilogue warp (warp - 4)
+    // One lane per warp.  It keeps G and U of its epilogue warp's rows kAhead chunks ahead (TMA loads
+    // into the ring) and writes each chunk back once the epilogue warp has turned it into dG, dU in
+    // place (TMA stores), so that the epilogue warp itself never issues or awaits a copy.
+    if constexpr (MODE == kDgrad1) {
+      if (lane == 0) {
+        const int ew = warp - 6;
+        const int quarter = (ew + 2) & 3;
+        uint8_t* stg = smem + TR::kStagingOffset + ew * TR::kStagingPerWarp;
+        uint64_t* full = epi_bar + kRing * ew;
+        uint64_t* staged = staged_bar + kRing * ew;
+        ChunkCursor<MODE> ld, st;
+        ld.start(p, total, n_nt, n_mt, quarter);
+        st.start(p, total, n_nt, n_mt, quarter);
+        int fetched = 0, stored = 0;
+        bool ok = true;
+        while (st.tile < total && ok) {
+          // A slot is refilled only after the store that last read it has drained: when chunk
+          // `fetched` <= stored + 2 is fetched, that store (chunk fetched - 5) is at least three
+          // bulk groups old, hence wait_group.read 1.
+          while (fetched < stored + kAhead && ld.tile < total) {
+            const int slot = fetched % kRing;
+            uint8_t* buf = stg + slot * 2 * kBf16ChunkBytes;
+            tc::bulk_wait_read<1>();
+            tc::mbar_expect_tx(&full[slot], 2 * kBf16ChunkBytes);
+            tc::tma_load_2d(buf, &tmC1, &full[slot], ld.col(), ld.row0);
+            tc::tma_load_2d(buf + kBf16ChunkBytes, &tmC1, &full[slot], p.f + ld.col(), ld.row0);
+            ++fetched;
+            ld.next(p, total, n_nt, n_mt, quarter);
+          }
+          const int slot = stored % kRing;
+          uint8_t* buf = stg + slot * 2 * kBf16ChunkBytes;
+          if (!tc::mbar_wait(&staged[slot], (stored / kRing) & 1, abort)) { report_timeout(p, abort, 6); ok = false; break; }
+          tc::tma_store_2d(&tmC0, buf, st.col(), st.row0);
+          tc::tma_store_2d(&tmC0, buf + kBf16ChunkBytes, p.f + st.col(), st.row0);
+          tc::bulk_commit();
+          ++stored;
+          st.next(p, total, n_nt, n_mt, quarter);
+        }
+        if (!ok)
+          for (int i = 0; i < 200; ++i) __nanosleep(1000);   // let loads already in flight land
+        tc::bulk_wait<0>();
+      }
+    }
   } else {
     // ------------------------------------------------------------ epilogue (warps 2..5)
     // Warp w owns TMEM lanes [32*(w%4), +32) = 32 rows of the tile.  Results are rounded,
@@ -313,10 +390,10 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     const int quarter = warp & 3;
     const int ew = warp - 2;
     uint8_t* stg = smem + TR::kStagingOffset + ew * TR::kStagingPerWarp;
-    constexpr int kRing = 5, kAhead = 3;               // dgrad1: (G, U) chunk buffers, prefetch distance
-    uint64_t* my_bar = epi_bar + kRing * ew;
+    uint64_t* my_bar = epi_bar + kRing * ew;           // dgrad1: chunk n of this warp's stream is in slot n % kRing
+    uint64_t* my_staged = staged_bar + kRing * ew;
     int gchunk = 0;                                    // chunks this warp has staged so far (ring position)
-    (void)my_bar;
+    (void)my_bar; (void)my_staged;
     int local = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
@@ -351,24 +428,8 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
       ++local;
       const int row0 = c.mt * BM + quarter * 32;       // first row of this warp (row tiles: permuted row)
 
-      // dgrad1: chunk j of this tile (global chunk gchunk + j) lands in ring slot (gchunk + j) % kRing.
-      // A slot is refilled only after the store that last read it has drained: that store is
-      // at least two bulk groups old whenever a fetch is issued, hence wait_group.read 1.
       int nch = 0;
-      auto fetch_gu = [&](int j) {
-        const int slot = (gchunk + j) % kRing;
-        uint8_t* buf = stg + slot * 2 * kBf16ChunkBytes;
-        const int col = c.nt * BN + j * kChunk;
-        tc::bulk_wait_read<1>();
-        tc::mbar_expect_tx(&my_bar[slot], 2 * kBf16ChunkBytes);
-        tc::tma_load_2d(buf, &tmC1, &my_bar[slot], col, row0);
-        tc::tma_load_2d(buf + kBf16ChunkBytes, &tmC1, &my_bar[slot], p.f + col, row0);
-      };
-      if constexpr (MODE == kDgrad1) {                 // fetch the first chunks while the MMAs still run
-        nch = min(BN / kChunk, (p.f - c.nt * BN) / kChunk);
-        if (lane == 0)
-          for (int j = 0; j < kAhead && j < nch; ++j) fetch_gu(j);
-      }
+      if constexpr (MODE == kDgrad1) nch = min(BN / kChunk, (p.f - c.nt * BN) / kChunk);
       if (!tc::mbar_wait(&tmem_full[acc], acc_phase, abort)) {
         if (lane == 0) report_timeout(p, abort, 4);
         break;
@@ -392,19 +453,19 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
             u[i] = __uint_as_float(ru[i]);
             a[i] = g[i] * sigmoid_fast(g[i]) * u[i];
           }
-          if (lane == 0) tc::bulk_wait_read<0>();      // the previous chunk's stores have drained the tiles
+          // lanes 0, 1, 2 each own one of the three stores (G, U, A), so the stores are issued and
+          // their shared-memory reads awaited side by side
+          if (lane < 3) tc::bulk_wait_read<0>();       // the previous chunk's stores have drained the tiles
           __syncwarp();
           stage_row_bf16(stg, lane, g);
           stage_row_bf16(stg + kBf16ChunkBytes, lane, u);
           stage_row_bf16(stg + 2 * kBf16ChunkBytes, lane, a);
           tc::fence_proxy_async();
           __syncwarp();
-          if (lane == 0) {
-            tc::tma_store_2d(&tmC0, stg, feat, row0);
-            tc::tma_store_2d(&tmC0, stg + kBf16ChunkBytes, p.f + feat, row0);
-            tc::tma_store_2d(&tmC1, stg + 2 * kBf16ChunkBytes, feat, row0);
-            tc::bulk_commit();
-          }
+          if (lane == 0) tc::tma_store_2d(&tmC0, stg, feat, row0);
+          else if (lane == 1) tc::tma_store_2d(&tmC0, stg + kBf16ChunkBytes, p.f + feat, row0);
+          else if (lane == 2) tc::tma_store_2d(&tmC1, stg + 2 * kBf16ChunkBytes, feat, row0);
+          if (lane < 3) tc::bulk_commit();
         }
       } else if constexpr (MODE == kFwd2 || MODE == kDgrad2) {
 #pragma unroll 1
@@ -432,11 +493,9 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
       } else if constexpr (MODE == kDgrad1) {
 #pragma unroll 1
         for (int ch = 0; ch < nch; ++ch) {
-          const int col = c.nt * BN + ch * kChunk;
           const int slot = (gchunk + ch) % kRing;
           const uint32_t slot_phase = ((gchunk + ch) / kRing) & 1;
           uint8_t* buf = stg + slot * 2 * kBf16ChunkBytes;
-          if (lane == 0 && ch + kAhead < nch) fetch_gu(ch + kAhead);
           uint32_t rr[32];
           tc::tmem_ld_32x32(t_row + ch * kChunk, rr);
           tc::tmem_ld_wait();
@@ -460,11 +519,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
           stage_row_bf16(buf + kBf16ChunkBytes, lane, du);
           tc::fence_proxy_async();
           __syncwarp();
-          if (lane == 0) {
-            tc::tma_store_2d(&tmC0, buf, col, row0);
-            tc::tma_store_2d(&tmC0, buf + kBf16ChunkBytes, p.f + col, row0);
-            tc::bulk_commit();
-          }
+          if (lane == 0) tc::mbar_arrive(&my_staged[slot]);   // the operand mover stores the chunk
         }
         gchunk += nch;
         if (!ok) break;
@@ -501,7 +556,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     }
     if (!ok && lane == 0)
       for (int i = 0; i < 200; ++i) __nanosleep(1000);  // let loads already in flight land before the CTA retires
-    if (lane == 0) tc::bulk_wait<0>();                 // every store has left shared memory and is complete
+    if (lane < 3) tc::bulk_wait<0>();                  // every store has left shared memory and is complete
     __syncwarp();
   }
 
@@ -566,7 +621,7 @@ int launch(unipool_ctx* ctx, int phase, const CUtensorMap& tmA, const CUtensorMa
   PhaseTimer pt(ctx, phase, 1, s);
   auto kern = grouped_gemm_tc_kernel<MODE>;
   UP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemTotal));
-  kern<<<ctx->sm_count, kThreads, kSmemTotal, s>>>(tmA, tmB, tmC0, tmC1, p);
+  kern<<<ctx->sm_count, Traits<MODE>::kThreads, kSmemTotal, s>>>(tmA, tmB, tmC0, tmC1, p);
   UP_LAUNCH_CHECK();
   return UNIPOOL_OK;
 }
