@@ -23,7 +23,7 @@ constexpr int BM = 128;          // rows of an output tile (TMEM lanes)
 constexpr int BN = 256;          // columns of an output tile (one tcgen05.mma of N = 256)
 constexpr int BK = 64;           // k-block: 64 bf16 = one 128-byte swizzle row
 constexpr int kThreads = 192;           // producer warp, MMA warp, four epilogue warps
-constexpr int kThreadsIo = 320;         // dgrad1: plus four warps that move the epilogue's operands
+constexpr int kThreadsIo = 448;         // dgrad1: eight epilogue warps plus four warps that move their operands
 constexpr int kEpiWarps = 4;
 constexpr uint32_t kABytes = BM * BK * 2;
 constexpr uint32_t kBBytes = BN * BK * 2;
@@ -220,7 +220,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { tc::mbar_init(&full_bar[s], 1); tc::mbar_init(&empty_bar[s], 1); }
-    for (int a = 0; a < 2; ++a) { tc::mbar_init(&tmem_full[a], 1); tc::mbar_init(&tmem_empty[a], kEpiWarps); }
+    for (int a = 0; a < 2; ++a) { tc::mbar_init(&tmem_full[a], 1); tc::mbar_init(&tmem_empty[a], MODE == kDgrad1 ? 2 * kEpiWarps : kEpiWarps); }
     for (int i = 0; i < 5 * kEpiWarps; ++i) { tc::mbar_init(&epi_bar[i], 1); tc::mbar_init(&staged_bar[i], 1); }
     *abort = 0;
     tc::fence_barrier_init();
@@ -337,14 +337,14 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
         if (ok) tc::umma_commit(&tmem_full[acc]);        // accumulator complete
       }
     }
-  } else if (warp >= 6) {
+  } else if (MODE == kDgrad1 && warp >= 2 + 2 * kEpiWarps) {
     // ------------------------------------------------------------ dgrad1: operand mover of epilogue warp (warp - 4)
     // One lane per warp.  It keeps G and U of its epilogue warp's rows kAhead chunks ahead (TMA loads
     // into the ring) and writes each chunk back once the epilogue warp has turned it into dG, dU in
     // place (TMA stores), so that the epilogue warp itself never issues or awaits a copy.
     if constexpr (MODE == kDgrad1) {
       if (lane == 0) {
-        const int ew = warp - 6;
+        const int ew = warp - (2 + 2 * kEpiWarps);
         const int quarter = (ew + 2) & 3;
         uint8_t* stg = smem + TR::kStagingOffset + ew * TR::kStagingPerWarp;
         uint64_t* full = epi_bar + kRing * ew;
@@ -387,8 +387,11 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     // Warp w owns TMEM lanes [32*(w%4), +32) = 32 rows of the tile.  Results are rounded,
     // staged in this warp's shared-memory tiles and leave through TMA stores; nothing
     // here synchronises with another warp except the two TMEM barriers.
+    // (dgrad1 has two epilogue warps per 32 lanes: they share one ring and take alternate chunks)
     const int quarter = warp & 3;
-    const int ew = warp - 2;
+    const int ew = (warp - 2) & 3;
+    const int half = (warp - 2) >> 2;
+    (void)half;
     uint8_t* stg = smem + TR::kStagingOffset + ew * TR::kStagingPerWarp;
     uint64_t* my_bar = epi_bar + kRing * ew;           // dgrad1: chunk n of this warp's stream is in slot n % kRing
     uint64_t* my_staged = staged_bar + kRing * ew;
@@ -493,6 +496,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
       } else if constexpr (MODE == kDgrad1) {
 #pragma unroll 1
         for (int ch = 0; ch < nch; ++ch) {
+          if (((gchunk + ch) & 1) != half) continue;    // the other warp of this quarter takes it
           const int slot = (gchunk + ch) % kRing;
           const uint32_t slot_phase = ((gchunk + ch) / kRing) & 1;
           uint8_t* buf = stg + slot * 2 * kBf16ChunkBytes;
