@@ -178,6 +178,7 @@ int route_bwd_tc_launch(unipool_ctx*, const void* x, int T, const float* W_r, fl
                         const float* coef, void* dx, float* dW_r, float* dsigma, cudaStream_t);
 int tc_operand_map(unipool_ctx*, void* out_tensor_map, const void* base, uint64_t cols, uint64_t rows,
                    uint32_t box_rows);
+int tc_f32_chunk_map(unipool_ctx*, void* out_tensor_map, const void* base, uint64_t cols, uint64_t rows);
 int router_bwd_gemms_tc(unipool_ctx*, const void* dz16, int Mp, const void* W16, const void* x, int T, int M,
                         void* dx, float* dW_r, cudaStream_t);
 int expert_fwd_simt(unipool_ctx*, const ExpertFwdArgs&, cudaStream_t);

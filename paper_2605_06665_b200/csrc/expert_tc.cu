@@ -747,6 +747,11 @@ int tc_operand_map(unipool_ctx* ctx, void* out, const void* base, uint64_t cols,
   return map_2d(ctx, static_cast<CUtensorMap*>(out), base, cols, rows, 64, box_rows);
 }
 
+// fp32 [rows, cols] map of 32 x 32 chunks with the 128-byte swizzle (epilogue-style stores)
+int tc_f32_chunk_map(unipool_ctx* ctx, void* out, const void* base, uint64_t cols, uint64_t rows) {
+  return map_chunk(ctx, static_cast<CUtensorMap*>(out), base, cols, rows, kMapF32Chunk);
+}
+
 // Router backward GEMMs (bf16 mode).  dz16 [T, Mp] bf16 (Mp = M rounded up to 64, pad columns
 // zero), W16 [M, d] bf16, x [T, d] bf16:
 //   dx [T, d] bf16 += dz16 W16        (row tiles, one group, TMA add-reduce into dx)

@@ -73,11 +73,12 @@ __device__ __forceinline__ void route_timeout(const RouteParams& p, volatile int
 template <int KMAX>
 __global__ void __launch_bounds__(kThreads, 1)
 route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW,
-                const RouteParams p) {
+                const __grid_constant__ CUtensorMap tmZ, const RouteParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t stage_bytes = kXBytes + p.w_bytes;
-  uint8_t* tail = smem + (size_t)p.stages * stage_bytes;
+  uint8_t* zstage = smem + (size_t)p.stages * stage_bytes;        // [4 warps][2] 32 x 32 fp32 tiles of z
+  uint8_t* tail = zstage + 4 * 2 * 4096;
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(tail);
   uint64_t* empty_bar = full_bar + kMaxStages;
   uint64_t* tmem_full = empty_bar + kMaxStages;
@@ -86,6 +87,7 @@ route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   int* last_flag = const_cast<int*>(abort) + 1;
   int* hist = reinterpret_cast<int*>(tail + 128);                  // [M]
   float* wsum = reinterpret_cast<float*>(hist + UNIPOOL_MAX_EXPERTS);   // [4][M] per-warp score sums
+  float* sbias = wsum + 4 * p.M;                                         // [ceil32(M)] logit bias (zeros without one)
 
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
   const int M = p.M;
@@ -101,6 +103,7 @@ route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     tc::tma_prefetch_desc(&tmW);
   }
   for (int i = threadIdx.x; i < M; i += blockDim.x) hist[i] = 0;
+  for (int i = threadIdx.x; i < (M + 31) / 32 * 32; i += blockDim.x) sbias[i] = (p.bias && i < M) ? p.bias[i] : 0.f;
   if (warp == 5) {
     tc::tmem_alloc(tmem_ptr, p.tmem_cols);
     tc::tmem_relinquish();
@@ -174,10 +177,14 @@ route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     tc::tc_fence_after_sync();
     const uint32_t t_row = tmem_base + (static_cast<uint32_t>(warp * 32) << 16);
     if (ok) {
-      // pass 1: logits (+ bias) -> z_saved, squared norm
+      // pass 1: logits (+ bias) -> z_saved, squared norm.  With a 16-byte row pitch (M % 4 == 0) the
+      // 32 x 32 chunk is staged in shared memory (128-byte swizzle, conflict-free) and leaves by a
+      // TMA store, which clips it at M columns and T rows.
       float ss = 0.f;
       float* zrow = p.z_saved + (int64_t)t * M;
       const bool vec = (M & 3) == 0;
+      uint8_t* my_stage = zstage + warp * 2 * 4096;
+      int nstore = 0;
       for (int c0 = 0; c0 < M; c0 += 32) {
         uint32_t rr[32];
         tc::tmem_ld_32x32(t_row + c0, rr);
@@ -185,21 +192,27 @@ route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         float z[32];
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
-          const int e = c0 + i;
-          z[i] = e < M ? __uint_as_float(rr[i]) + (p.bias ? __ldg(p.bias + e) : 0.f) : 0.f;
+          z[i] = c0 + i < M ? __uint_as_float(rr[i]) + sbias[c0 + i] : 0.f;
           ss = fmaf(z[i], z[i], ss);
         }
-        if (live) {
-          if (vec) {
+        if (vec) {
+          uint8_t* buf = my_stage + (nstore++ & 1) * 4096;
+          if (lane == 0) tc::bulk_wait_read<1>();       // the store issued two chunks ago has drained `buf`
+          __syncwarp();
 #pragma unroll
-            for (int q = 0; q < 8; ++q)
-              if (c0 + 4 * q < M)
-                *reinterpret_cast<float4*>(zrow + c0 + 4 * q) = make_float4(z[4 * q], z[4 * q + 1], z[4 * q + 2], z[4 * q + 3]);
-          } else {
-#pragma unroll
-            for (int i = 0; i < 32; ++i)
-              if (c0 + i < M) zrow[c0 + i] = z[i];
+          for (int q = 0; q < 8; ++q)
+            *reinterpret_cast<float4*>(buf + lane * 128 + ((q ^ (lane & 7)) << 4)) =
+                make_float4(z[4 * q], z[4 * q + 1], z[4 * q + 2], z[4 * q + 3]);
+          tc::fence_proxy_async();
+          __syncwarp();
+          if (lane == 0) {
+            tc::tma_store_2d(&tmZ, buf, c0, blockIdx.x * kTile + warp * 32);
+            tc::bulk_commit();
           }
+        } else if (live) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i)
+            if (c0 + i < M) zrow[c0 + i] = z[i];
         }
       }
       const float n = sqrtf(ss);
@@ -218,26 +231,27 @@ route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
           const int e = c0 + i;
-          float s = 0.f;
-          if (e < M) {
-            const float z = __uint_as_float(rr[i]) + (p.bias ? __ldg(p.bias + e) : 0.f);
-            s = scale * fmaxf(z, 0.f);
-            float key = s;
-            if (!(key == key)) key = -FLT_MAX;            // NaN scores sort last but stay selectable
-            if (key > tv[KMAX - 1]) {
-              // insert behind every entry that is >= key (equal keys keep the lower index in
-              // front), then shift the displaced entries down by one
-              float cv = key;
-              int ci = e;
-              bool moved = false;
+          const float z = __uint_as_float(rr[i]) + sbias[e < M ? e : 0];
+          const float s = e < M ? scale * fmaxf(z, 0.f) : 0.f;
+          float key = s == s ? s : -FLT_MAX;              // NaN scores sort last but stay selectable
+          if (e >= M) key = -INFINITY;                    // never selected
+          // Insert behind every entry that is >= key (equal keys keep the lower index in front) and
+          // shift the displaced entries down by one.  For short lists this is a fixed sequence of
+          // selects; long lists test the last entry first, since most scores do not enter.
+          if (KMAX <= 2 || key > tv[KMAX - 1]) {
+            float cv = key;
+            int ci = e;
+            bool moved = false;
 #pragma unroll
-              for (int j = 0; j < KMAX; ++j) {
-                if (moved || cv > tv[j]) {
-                  const float fv = tv[j]; tv[j] = cv; cv = fv;
-                  const int fi = ti[j]; ti[j] = ci; ci = fi;
-                  moved = true;
-                }
-              }
+            for (int j = 0; j < KMAX; ++j) {
+              const bool sw = moved || cv > tv[j];
+              const float fv = tv[j];
+              const int fi = ti[j];
+              tv[j] = sw ? cv : fv;
+              ti[j] = sw ? ci : fi;
+              cv = sw ? fv : cv;
+              ci = sw ? fi : ci;
+              moved = sw;
             }
           }
           sv[i] = live ? s : 0.f;
@@ -269,6 +283,7 @@ route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         }
       }
     }
+    if (lane == 0) tc::bulk_wait<0>();                   // the z tiles have left shared memory
     tc::tc_fence_before_sync();
     // the four epilogue warps publish the tile's statistics (named barrier 1: 128 threads)
     asm volatile("bar.sync 1, 128;" ::: "memory");
@@ -280,18 +295,27 @@ route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     asm volatile("bar.sync 1, 128;" ::: "memory");
     if (threadIdx.x == 0) *last_flag = atomicAdd(p.ticket, 1u) == gridDim.x - 1 ? 1 : 0;
     asm volatile("bar.sync 1, 128;" ::: "memory");
-    if (*last_flag) {                     // the CTA that arrives last adds the tiles up, in tile order
+    if (*last_flag) {                     // the CTA that arrives last adds the tiles up
+      // warp w sums the tiles b = w, w + 4, ... (independent loads), then the four partial sums of an
+      // expert are added in warp order: the result does not depend on which CTA came last
       __threadfence();
-      for (int i = threadIdx.x; i < M; i += kTile) {
+      double* dsum = reinterpret_cast<double*>(zstage);  // [4][M] in the z staging tiles (they have drained)
+      int* csum = reinterpret_cast<int*>(zstage + 4 * UNIPOOL_MAX_EXPERTS * sizeof(double));   // [4][M]
+      for (int i = lane; i < M; i += 32) {
         int cnt = 0;
         double sum = 0.0;
 #pragma unroll 8
-        for (int b = 0; b < (int)gridDim.x; ++b) {
+        for (int b = warp; b < (int)gridDim.x; b += 4) {
           cnt += __ldcg(&p.part_counts[(int64_t)b * M + i]);
           sum += (double)__ldcg(&p.part_sums[(int64_t)b * M + i]);
         }
-        p.counts_out[i] = cnt;
-        p.sum_out[i] = (float)sum;
+        csum[warp * M + i] = cnt;
+        dsum[warp * M + i] = sum;
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      for (int i = threadIdx.x; i < M; i += kTile) {
+        p.counts_out[i] = (csum[i] + csum[M + i]) + (csum[2 * M + i] + csum[3 * M + i]);
+        p.sum_out[i] = (float)((dsum[i] + dsum[M + i]) + (dsum[2 * M + i] + dsum[3 * M + i]));
       }
       if (threadIdx.x == 0) *p.ticket = 0u;
     }
@@ -395,7 +419,7 @@ int route_tc_launch(unipool_ctx* ctx, const void* x, int T, const float* W_r, fl
   p.status = ctx->ws.status;
   p.w_bytes = (uint32_t)((M + 127) / 128) * 16384u;
   const uint32_t stage_bytes = kXBytes + p.w_bytes;
-  const uint32_t tail_bytes = 128 + UNIPOOL_MAX_EXPERTS * 4 + 4 * M * 4;
+  const uint32_t tail_bytes = 4 * 2 * 4096 + 128 + UNIPOOL_MAX_EXPERTS * 4 + 4 * M * 4 + (M + 31) / 32 * 32 * 4;
   const uint32_t budget = 227 * 1024 - 1024 - tail_bytes;
   p.stages = (int)(budget / stage_bytes);
   if (p.stages > kMaxStages) p.stages = kMaxStages;
@@ -408,7 +432,12 @@ int route_tc_launch(unipool_ctx* ctx, const void* x, int T, const float* W_r, fl
     PhaseTimer pt(ctx, UNIPOOL_PH_ROUTE_LOGITS, 1, s);
     if ((rc = router_split_launch(ctx, W_r, M, s)) != UNIPOOL_OK) return rc;
   }
-  CUtensorMap tmX, tmW;
+  CUtensorMap tmX, tmW, tmZ;
+  if ((M & 3) == 0) {
+    if ((rc = tc_f32_chunk_map(ctx, &tmZ, z_saved, M, T)) != UNIPOOL_OK) return rc;
+  } else {
+    tmZ = CUtensorMap{};                 // not used: rows of z are not 16-byte aligned, plain stores instead
+  }
   if ((rc = tc_operand_map(ctx, &tmX, x, d, T, kTile)) != UNIPOOL_OK) return rc;
   if ((rc = tc_operand_map(ctx, &tmW, ctx->ws.w_split, d, (uint64_t)3 * M, 128)) != UNIPOOL_OK) return rc;
   PhaseTimer pt(ctx, UNIPOOL_PH_ROUTE_SELECT, 1, s);
@@ -416,10 +445,10 @@ int route_tc_launch(unipool_ctx* ctx, const void* x, int T, const float* W_r, fl
   const int grid = (T + kTile - 1) / kTile;
   if (k <= 2) {
     UP_CUDA(cudaFuncSetAttribute(route_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    route_tc_kernel<2><<<grid, kThreads, smem, s>>>(tmX, tmW, p);
+    route_tc_kernel<2><<<grid, kThreads, smem, s>>>(tmX, tmW, tmZ, p);
   } else {
     UP_CUDA(cudaFuncSetAttribute(route_tc_kernel<UNIPOOL_MAX_TOPK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    route_tc_kernel<UNIPOOL_MAX_TOPK><<<grid, kThreads, smem, s>>>(tmX, tmW, p);
+    route_tc_kernel<UNIPOOL_MAX_TOPK><<<grid, kThreads, smem, s>>>(tmX, tmW, tmZ, p);
   }
   UP_LAUNCH_CHECK();
   return UNIPOOL_OK;

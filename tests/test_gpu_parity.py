@@ -160,6 +160,7 @@ def test_small_fp32_shapes(kw, T):
     (dict(dtype="bf16", d=256, f=384, M=16, k=2), 1000),
     (dict(dtype="bf16", d=128, f=128, M=384, k=8, zipf_beta=0.4), 600),
     (dict(dtype="bf16", d=256, f=256, M=12, k=2, private=4, L=3), 520),
+    (dict(dtype="bf16", d=128, f=128, M=10, k=3), 333),     # logit rows that are not 16-byte aligned
 ])
 def test_small_bf16_shapes(kw, T):
     cfg = small_cfg(**kw)
