@@ -185,6 +185,18 @@ def run_ours(args):
         xL_host.copy_(st.x[L], non_blocking=True)
         loss_host.copy_(st.loss, non_blocking=True)
 
+    if args.graph:                           # one CUDA graph per step variant: same kernels, one launch
+        g_dev = st.capture_step(x0, up, accumulate=False)
+        g_e2e = st.capture_step(x0_host, up_host, accumulate=False)
+        eager_step = device_step
+        device_step = g_dev.replay
+
+        def e2e_step():
+            g_e2e.replay()
+            xL_host.copy_(st.x[L], non_blocking=True)
+            loss_host.copy_(st.loss, non_blocking=True)
+    else:
+        eager_step = device_step
     for _ in range(max(args.warmup, 3)):
         device_step()
     st.ctx.check_status()
@@ -203,7 +215,7 @@ def run_ours(args):
 
     # per-kernel durations, measured live with CUDA events on the launch stream
     st.ctx.profile_enable(True)
-    timed(device_step, args.steps)
+    timed(eager_step, args.steps)
     prof = st.ctx.profile_read()
     st.ctx.profile_enable(False)
 
@@ -281,7 +293,7 @@ def run_ours(args):
         "vs_baseline": None, "dtype": cfg["dtype"], "data": "synthetic",
         "config": {"workload": args.workload, "layers": L, "d_model": d, "d_ff": f, "pool_experts": M, "top_k": k,
                    "tokens_per_gpu": T, "layout": "private" if cfg["private"] else "shared_pool",
-                   "deferred_wgrad": bool(st.deferred_wgrad),
+                   "deferred_wgrad": bool(st.deferred_wgrad), "cuda_graph": bool(args.graph),
                    "l2": "working set per step (weights + saved activations, several GB) exceeds the 126 MB L2",
                    "norm_router_c": c_val},
         "clocks": clocks,
@@ -378,6 +390,8 @@ def main():
                          "backward instead of contracting all layers' rows per expert in one pass at the end")
     ap.add_argument("--cpu-tokens", type=int, default=16384, help="token sample of the CPU-oracle baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", dest="graph", action="store_false",
+                    help="issue every library call of a step eagerly instead of replaying one CUDA graph")
     ap.add_argument("--kernels-only", action="store_true",
                     help="run warm-up and timed steps only and print no result (for runs under a profiler)")
     args = ap.parse_args()

@@ -175,5 +175,20 @@ class UniPoolStack:
             self.zero_router_grad()
         return self.backward(upstream, T, accumulate=accumulate)
 
+    def capture_step(self, x0=None, upstream=None, accumulate=True):
+        """Records one whole step (the library calls of ``step`` with these tensors) into a CUDA graph
+        and returns it; ``graph.replay()`` then issues the step with one launch.  Every call of the
+        path is asynchronous on the stream and allocates nothing, so the recording holds exactly the
+        kernels and copies an eager step issues."""
+        side = torch.cuda.Stream(self.device)
+        side.wait_stream(torch.cuda.current_stream(self.device))
+        with torch.cuda.stream(side):                       # one eager pass first: lazy set-up happens here
+            self.step(x0, upstream, accumulate=accumulate)
+        torch.cuda.current_stream(self.device).wait_stream(side)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            self.step(x0, upstream, accumulate=accumulate)
+        return graph
+
     def close(self):
         self.ctx.close()

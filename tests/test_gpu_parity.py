@@ -239,6 +239,34 @@ def test_fp32_router_weights_in_bf16_mode():
     st.close()
 
 
+def test_cuda_graph_replay_matches_eager_step():
+    """A step recorded into a CUDA graph issues the same kernels: replaying it reproduces the eager
+    step's outputs and gradients bit for bit (overwriting pass, deterministic kernels)."""
+    import torch
+    cfg = small_cfg(dtype="bf16", d=256, f=384, M=16, k=2, L=3)
+    T = 900
+    inputs = synth.make_inputs(cfg, seed=9, T=T)
+    x0 = torch.from_numpy(inputs["x0"]).cuda().bfloat16()
+    up = torch.from_numpy(inputs["upstream"]).cuda().bfloat16()
+    st = build_stack(cfg, inputs, T=T, deferred_wgrad=True)
+    st.step(x0, up, accumulate=False)
+    torch.cuda.synchronize()
+    ref = [t.clone() for t in (st.x[cfg["L"]], st.dW_gu, st.dW_down, st.dW_r, st.loss, st.idx)]
+    graph = st.capture_step(x0, up, accumulate=False)
+    for t in (st.x, st.dW_gu, st.dW_down, st.dW_r):
+        t.fill_(1.0)
+    graph.replay()
+    graph.replay()
+    torch.cuda.synchronize()
+    st.ctx.check_status()
+    got = (st.x[cfg["L"]], st.dW_gu, st.dW_down, st.dW_r, st.loss, st.idx)
+    for a, b in zip(ref[:3] + ref[5:], got[:3] + got[5:]):
+        assert torch.equal(a, b)
+    assert rel_max(to_np(got[3]), to_np(ref[3])) < 1e-5             # fp32 add-reduce order may differ
+    assert torch.allclose(ref[4], got[4], rtol=1e-6)
+    st.close()
+
+
 def test_empty_batch():
     import torch
     cfg = small_cfg()
