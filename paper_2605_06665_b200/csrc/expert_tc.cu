@@ -12,6 +12,8 @@
 // UNIPOOL_ERR_TIMEOUT in the status word, all roles leave, TMEM is released.
 #include <cuda.h>
 
+#include <cstdlib>
+
 #include "common.cuh"
 #include "tc_ptx.cuh"
 
@@ -572,6 +574,214 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
   }
 }
 
+// ---------------------------------------------------------------- weight gradient on CTA pairs
+// dW[e] (+)= P_e^T Q_e with one tcgen05.mma.cta_group::2 of M = 256, N = 256 per K = 16: the two CTAs
+// of a cluster own rows [0,128) and [128,256) of the 256 x 256 output tile (their own TMEM), each
+// loads its 128 columns of P (A operand) and HALF of the 256 columns of Q (B operand), so a CTA
+// moves 32 KB per k-block for the work that took 48 KB, and six stages fit instead of four.  The
+// even CTA issues the MMAs; every TMA load counts its bytes on the even CTA's mbarrier (plain
+// loads, no multicast); tcgen05.commit arrives on the stage / accumulator barriers of both CTAs.
+constexpr int kPairStages = 6;
+constexpr uint32_t kPairHalfBytes = 128 * BK * 2;            // 128 (M or N) x 64 (K) bf16
+constexpr uint32_t kPairStageBytes = 2 * kPairHalfBytes;
+static_assert(kPairStages * kPairStageBytes + kEpiWarps * 8192 == kBarOffset, "shared-memory budget");
+
+__device__ __forceinline__ int wgrad_kblocks(const GemmParams& p, int e) {
+  int kb = 0;
+  for (int l = 0; l < p.n_layers; ++l) {
+    const int32_t* off = p.offsets + (int64_t)l * (p.n_experts + 1);
+    kb += (off[e + 1] - off[e]) / BK;
+  }
+  return kb;
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+wgrad_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                  const __grid_constant__ CUtensorMap tmC0, const GemmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + kBarOffset);
+  uint64_t* empty_bar = full_bar + kPairStages;
+  uint64_t* tmem_full = empty_bar + kPairStages;
+  uint64_t* tmem_empty = tmem_full + 2;
+  uint32_t* tmem_ptr = reinterpret_cast<uint32_t*>(tmem_empty + 2);
+  volatile int* abort = reinterpret_cast<volatile int*>(tmem_ptr + 1);
+
+  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+  const int rank = (int)tc::cluster_ctarank();               // 0 = leader
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kPairStages; ++s) { tc::mbar_init(&full_bar[s], 1); tc::mbar_init(&empty_bar[s], 1); }
+    for (int a = 0; a < 2; ++a) { tc::mbar_init(&tmem_full[a], 1); tc::mbar_init(&tmem_empty[a], 2 * kEpiWarps); }
+    *abort = 0;
+    tc::fence_barrier_init();
+    tc::tma_prefetch_desc(&tmA);
+    tc::tma_prefetch_desc(&tmB);
+    tc::tma_prefetch_desc(&tmC0);
+  }
+  if (warp == 1) {
+    tc::tmem_alloc_pair(tmem_ptr, 512);
+    tc::tmem_relinquish_pair();
+  }
+  tc::tc_fence_before_sync();
+  __syncthreads();
+  tc::cluster_sync();                                        // both CTAs' barriers exist before any remote use
+  tc::tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_ptr;
+
+  const int n_mt = (p.Mdim + 255) / 256, n_nt = (p.Ndim + 255) / 256;
+  const int per_e = n_mt * n_nt;
+  const int total = p.n_experts * per_e;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer (one in each CTA)
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = pair; tile < total && ok; tile += n_pairs) {
+        const int e = tile / per_e, rem = tile % per_e, mt = rem / n_nt, nt = rem % n_nt;
+        const int kblocks = wgrad_kblocks(p, e);
+        int layer = 0, r = p.offsets[e], r_end = p.offsets[e + 1];
+        for (int kb = 0; kb < kblocks; ++kb) {
+          if (!tc::mbar_wait(&empty_bar[stage], phase ^ 1u, abort)) { report_timeout(p, abort, 21); ok = false; break; }
+          while (r >= r_end) {                          // next layer that has rows for this expert
+            ++layer;
+            const int32_t* off = p.offsets + (int64_t)layer * (p.n_experts + 1);
+            r = off[e];
+            r_end = off[e + 1];
+          }
+          const int grow = layer * p.layer_stride_rows + r;
+          uint8_t* sA = smem + stage * kPairStageBytes;
+          uint8_t* sB = sA + kPairHalfBytes;
+          if (rank == 0) tc::mbar_expect_tx(&full_bar[stage], 2 * kPairStageBytes);   // both CTAs' bytes
+#pragma unroll
+          for (int i = 0; i < 2; ++i) {
+            tc::tma_load_2d_pair(sA + i * kMnBlockBytes, &tmA, &full_bar[stage], mt * 256 + rank * 128 + 64 * i, grow);
+            tc::tma_load_2d_pair(sB + i * kMnBlockBytes, &tmB, &full_bar[stage], nt * 256 + rank * 128 + 64 * i, grow);
+          }
+          r += BK;
+          if (++stage == kPairStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok)
+        for (int i = 0; i < 200; ++i) __nanosleep(1000);
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer (leader CTA only)
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = tc::instr_desc_bf16(256, true, true, 256);
+      constexpr uint32_t kstep = (16 * 128) >> 4;             // descriptor units per K = 16 (MN-major)
+      int stage = 0;
+      uint32_t phase = 0;
+      int local = 0;
+      bool ok = true;
+      for (int tile = pair; tile < total && ok; tile += n_pairs) {
+        const int kblocks = wgrad_kblocks(p, tile / per_e);
+        if (kblocks == 0) continue;
+        const int acc = local & 1;
+        const uint32_t acc_phase = (local >> 1) & 1;
+        ++local;
+        if (!tc::mbar_wait(&tmem_empty[acc], acc_phase ^ 1u, abort)) { report_timeout(p, abort, 22); break; }
+        tc::tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + acc * 256;
+        for (int kb = 0; kb < kblocks; ++kb) {
+          if (!tc::mbar_wait(&full_bar[stage], phase, abort)) { report_timeout(p, abort, 23); ok = false; break; }
+          tc::tc_fence_after_sync();
+          const uint32_t aaddr = tc::smem_u32(smem + stage * kPairStageBytes);
+          const uint64_t adesc = tc::smem_desc_sw128(aaddr, kMnBlockBytes, 1024);
+          const uint64_t bdesc = tc::smem_desc_sw128(aaddr + kPairHalfBytes, kMnBlockBytes, 1024);
+#pragma unroll
+          for (int j = 0; j < BK / 16; ++j)
+            tc::umma_bf16_pair(d_tmem, adesc + j * kstep, bdesc + j * kstep, idesc, (kb | j) != 0 ? 1u : 0u);
+          tc::umma_commit_pair(&empty_bar[stage], 3);           // frees the stage in both CTAs
+          if (++stage == kPairStages) { stage = 0; phase ^= 1u; }
+        }
+        if (ok) tc::umma_commit_pair(&tmem_full[acc], 3);       // accumulator complete, both CTAs
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue: this CTA's 128 rows of the tile
+    const int quarter = warp & 3;
+    uint8_t* stg = smem + kPairStages * kPairStageBytes + (warp - 2) * 8192;
+    int gchunk = 0, local = 0;
+    for (int tile = pair; tile < total; tile += n_pairs) {
+      const int e = tile / per_e, rem = tile % per_e, mt = rem / n_nt, nt = rem % n_nt;
+      const int m0 = mt * 256 + rank * 128 + quarter * 32;
+      const int grow = (p.expert_base + e) * p.Mdim + m0;
+      if (wgrad_kblocks(p, e) == 0) {
+        if (p.overwrite && m0 < p.Mdim) {               // no rows anywhere: the gradient of this tile is zero
+          if (lane == 0) tc::bulk_wait_read<0>();
+          __syncwarp();
+#pragma unroll
+          for (int q = 0; q < 8; ++q) *f32_piece(stg, lane, q) = make_uint4(0, 0, 0, 0);
+          tc::fence_proxy_async();
+          __syncwarp();
+          if (lane == 0) {
+            for (int ch = 0; ch < 256 / kChunk; ++ch) {
+              const int col = nt * 256 + ch * kChunk;
+              if (col < p.Ndim) tc::tma_store_2d(&tmC0, stg, col, grow);
+            }
+            tc::bulk_commit();
+            tc::bulk_wait_read<0>();
+          }
+          __syncwarp();
+        }
+        continue;
+      }
+      const int acc = local & 1;
+      const uint32_t acc_phase = (local >> 1) & 1;
+      ++local;
+      if (!tc::mbar_wait(&tmem_full[acc], acc_phase, abort)) {
+        if (lane == 0) report_timeout(p, abort, 24);
+        break;
+      }
+      tc::tc_fence_after_sync();
+      const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * 256;
+      if (m0 < p.Mdim) {
+#pragma unroll 1
+        for (int ch = 0; ch < 256 / kChunk; ++ch) {
+          const int col = nt * 256 + ch * kChunk;
+          if (col >= p.Ndim) break;
+          uint32_t rr[32];
+          tc::tmem_ld_32x32(t_row + ch * kChunk, rr);
+          tc::tmem_ld_wait();
+          uint8_t* buf = stg + (gchunk++ & 1) * kF32ChunkBytes;
+          if (lane == 0) tc::bulk_wait_read<1>();        // the store issued two chunks ago has drained `buf`
+          __syncwarp();
+#pragma unroll
+          for (int q = 0; q < 8; ++q)
+            *f32_piece(buf, lane, q) = make_uint4(rr[4 * q + 0], rr[4 * q + 1], rr[4 * q + 2], rr[4 * q + 3]);
+          tc::fence_proxy_async();
+          __syncwarp();
+          if (lane == 0) {
+            if (p.overwrite) tc::tma_store_2d(&tmC0, buf, col, grow);
+            else tc::tma_reduce_add_2d(&tmC0, buf, col, grow);
+            tc::bulk_commit();
+          }
+        }
+      }
+      tc::tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) {                                   // the leader's MMA thread waits for all eight warps
+        if (rank == 0) tc::mbar_arrive(&tmem_empty[acc]);
+        else tc::mbar_arrive_leader(&tmem_empty[acc]);
+      }
+    }
+    if (lane == 0) tc::bulk_wait<0>();
+    __syncwarp();
+  }
+
+  tc::tc_fence_before_sync();
+  __syncthreads();
+  tc::cluster_sync();                                        // neither CTA leaves while the other may still signal it
+  if (warp == 1) {
+    tc::tc_fence_after_sync();
+    tc::tmem_dealloc_pair(tmem_base, 512);
+  }
+}
+
 // ---------------------------------------------------------------- host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -630,6 +840,19 @@ int launch(unipool_ctx* ctx, int phase, const CUtensorMap& tmA, const CUtensorMa
   return UNIPOOL_OK;
 }
 
+// The pool weight gradient runs on CTA pairs (UNIPOOL_WGRAD_PAIR=0, a debugging aid, selects the
+// single-CTA kernel).
+int launch_wgrad(unipool_ctx* ctx, int phase, const CUtensorMap& tmP, const CUtensorMap& tmQ, const CUtensorMap& tmW,
+                 const GemmParams& p, cudaStream_t s) {
+  static const bool pair = [] { const char* v = getenv("UNIPOOL_WGRAD_PAIR"); return !(v && v[0] == '0'); }();
+  if (!pair || ctx->sm_count < 2) return launch<kWgrad>(ctx, phase, tmP, tmQ, tmW, tmW, p, s);
+  PhaseTimer pt(ctx, phase, 1, s);
+  UP_CUDA(cudaFuncSetAttribute(wgrad_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemTotal));
+  wgrad_pair_kernel<<<ctx->sm_count / 2 * 2, kThreads, kSmemTotal, s>>>(tmP, tmQ, tmW, p);
+  UP_LAUNCH_CHECK();
+  return UNIPOOL_OK;
+}
+
 int wgrad_pair(unipool_ctx* ctx, const PoolWgradArgs& a, cudaStream_t s) {
   const int d = ctx->cfg.d_model, f = ctx->cfg.d_ff, M = ctx->cfg.pool_size;
   const uint64_t rows = (uint64_t)(a.n_layers > 1 ? (int64_t)a.n_layers * a.layer_stride_rows : ctx->row_capacity);
@@ -648,13 +871,13 @@ int wgrad_pair(unipool_ctx* ctx, const PoolWgradArgs& a, cudaStream_t s) {
   if ((rc = map_2d(ctx, &tmQ, a.A, f, rows, 64, 64)) != UNIPOOL_OK) return rc;
   if ((rc = map_chunk(ctx, &tmW, a.dW_down, f, (uint64_t)M * d, kMapF32Chunk)) != UNIPOOL_OK) return rc;
   p.Mdim = d; p.Ndim = f;
-  if ((rc = launch<kWgrad>(ctx, UNIPOOL_PH_WGRAD_DOWN, tmP, tmQ, tmW, tmW, p, s)) != UNIPOOL_OK) return rc;
+  if ((rc = launch_wgrad(ctx, UNIPOOL_PH_WGRAD_DOWN, tmP, tmQ, tmW, p, s)) != UNIPOOL_OK) return rc;
   // dW_gu[e] [2f, d] (+)= dGU_e^T Xp_e
   if ((rc = map_2d(ctx, &tmP, a.dGU, 2 * f, rows, 64, 64)) != UNIPOOL_OK) return rc;
   if ((rc = map_2d(ctx, &tmQ, a.Xp, d, rows, 64, 64)) != UNIPOOL_OK) return rc;
   if ((rc = map_chunk(ctx, &tmW, a.dW_gu, d, (uint64_t)M * 2 * f, kMapF32Chunk)) != UNIPOOL_OK) return rc;
   p.Mdim = 2 * f; p.Ndim = d;
-  return launch<kWgrad>(ctx, UNIPOOL_PH_WGRAD_GU, tmP, tmQ, tmW, tmW, p, s);
+  return launch_wgrad(ctx, UNIPOOL_PH_WGRAD_GU, tmP, tmQ, tmW, p, s);
 }
 
 }  // namespace
