@@ -121,9 +121,8 @@ def run_ours(args):
     from paper_2605_06665_b200.stack import UniPoolStack
     import __graft_entry__ as entry
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2605_06665_b200 import dp
+    world, rank, local_rank = dp.env_world()
     if rank == 0:
         entry.build()
     torch.cuda.set_device(local_rank)
@@ -138,7 +137,7 @@ def run_ours(args):
     cfg = dict(synth.CONFIGS[args.workload])
     L, T, d, f, M, k = cfg["L"], cfg["T"], cfg["d"], cfg["f"], cfg["M"], cfg["k"]
     m = synth.router_width(cfg)
-    inputs = synth.make_inputs(cfg, seed=rank)
+    inputs = synth.make_inputs(cfg, seed=dp.shard_seed(rank))
     from paper_2605_06665_b200 import binding as B
     small = B.Context(B.make_config(64, 64, m, k, 1, 128, B.FP32, synth.EPS, 1.0), dev)
     c_val = small.calibrate_c(m, k, 100_000, seed=0)           # Alg. 1 on the device
@@ -168,12 +167,7 @@ def run_ours(args):
             fn()
         e1.record()
         sync_all()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return dp.max_over_ranks(e0.elapsed_time(e1), world, dev)
 
     def device_step():
         # the step's first weight-gradient contribution overwrites the fp32 pool gradient, so it
@@ -225,8 +219,8 @@ def run_ours(args):
     st.ctx.check_status()
 
     ms_step = ms_total / args.steps
-    value = world * T * L / (ms_step * 1e-3)
-    e2e_value = world * T * L / (ms_e2e / args.steps * 1e-3)
+    value = dp.whole_job_throughput(T * L, world, ms_step)
+    e2e_value = dp.whole_job_throughput(T * L, world, ms_e2e / args.steps)
     peaks = _peaks()
     R = T * k
     kernels = {}
