@@ -28,6 +28,11 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of a workload's dominant kernel,
+# from the ncu capture summarised in profiles/grouped_gemm_182m_slice_ncu.txt: the 182m_slice case (a quarter
+# of the experts and of the rows of one 182m layer) moved 165.6 + 79.8 MB; a full launch is four times that.
+NCU_TRAFFIC = {("182m", "expert_fwd_gu"): 4 * (165.58e6 + 79.81e6)}
+
 METRIC = "moe_layer_fwd_bwd_tokens_per_s"
 UNIT = "tokens/s"
 
@@ -276,6 +281,7 @@ def run_ours(args):
                         peak=peaks["bf16_tflops_sustained"], unit="TFLOP/s",
                         frac=dom["tflops"] / peaks["bf16_tflops_sustained"],
                         peak_source=peaks["source"] + " sustained", traffic=None, hbm_gbs=dom["gbs"])
+    roofline["traffic"] = NCU_TRAFFIC.get((args.workload, dominant))
     ceiling_s = sum(kernels[n]["ms_per_step"] * 1e-3 * kernels[n]["frac_of_ceiling"] for n in gemm_ms)
     total_gemm_flops = 18 * R * d * f * L
     gemm_time = sum(gemm_ms.values()) * 1e-3
