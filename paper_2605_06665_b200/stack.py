@@ -21,13 +21,17 @@ from . import binding as B
 
 class UniPoolStack:
     def __init__(self, L, d, f, M, k, T, dtype="bf16", private=0, c=1.0, eps=1e-6, alpha=1e-2,
-                 device="cuda", deferred_wgrad=False):
+                 device="cuda", deferred_wgrad=False, recompute=False):
         self.L, self.d, self.f, self.M, self.k, self.T = L, d, f, M, k, T
         self.private = private
         self.m = private if private else M                 # experts one router scores
         self.alpha = alpha
         self.c, self.eps = c, eps
-        self.deferred_wgrad = deferred_wgrad and not private
+        # recompute: keep only x_l and the routing state of a layer; its permuted activations are
+        # rebuilt in backward (MoE-layer activation recompute, App. D), so the weight gradient is
+        # taken layer by layer
+        self.recompute = recompute
+        self.deferred_wgrad = deferred_wgrad and not private and not recompute
         self.device = torch.device(device)
         self.tdtype = torch.bfloat16 if dtype == "bf16" else torch.float32
         self.cfg = B.make_config(d, f, M, k, L, T, B.BF16 if dtype == "bf16" else B.FP32, eps, c)
@@ -60,10 +64,11 @@ class UniPoolStack:
         self.row_of = e(L, T, k, dtype=i32)
         self.token_of = e(L, cap, dtype=i32)
         self.tile_expert = e(L, cap // B.ROW_ALIGN, dtype=i32)
-        self.Xp = e(L, cap, d)
-        self.GU = e(L, cap, 2 * f)
-        self.A = e(L, cap, f)
-        self.Yp = e(L, cap, d)
+        ns = 1 if recompute else L                         # layers whose permuted activations are kept
+        self.Xp = e(ns, cap, d)
+        self.GU = e(ns, cap, 2 * f)
+        self.A = e(ns, cap, f)
+        self.Yp = e(ns, cap, d)
         nb = L if self.deferred_wgrad else 1
         self.dYp = e(nb, cap, d)
         self.dGU = e(nb, cap, 2 * f)
@@ -74,6 +79,7 @@ class UniPoolStack:
         self.loss = torch.zeros(n_aux, dtype=f32, device=dev)
         self.coef = e(n_aux, self.m, dtype=f32)
         self.fbar = e(n_aux, self.m, dtype=f32)
+        self.fbar_lag = None                               # f-bar of the previous micro-batch (App. G)
 
     # ------------------------------------------------------------------ parameters
     def load(self, pool, routers):
@@ -93,6 +99,10 @@ class UniPoolStack:
     def base(self, l):
         return self.private * l if self.private else 0
 
+    def slot(self, l):
+        """Index of layer l's permuted activations (one shared slot when they are recomputed)."""
+        return 0 if self.recompute else l
+
     def zero_grad(self):
         self.dW_gu.zero_(); self.dW_down.zero_(); self.dW_r.zero_(); self.dsigma.zero_()
 
@@ -106,11 +116,17 @@ class UniPoolStack:
         bias = None if self.bias is None else self.bias[l]
         c.route(self.x[l], T, self.W_r[l], self.sigma[l], bias, self.m, self.idx[l], self.gate[l],
                 self.counts[l], self.score_sum[l], self.znorm[l], self.z[l])
+        self.permute_and_experts(l, T)
+        c.combine(self.Yp[self.slot(l)], self.row_of[l], self.gate[l], T, self.x[l], self.x[l + 1])
+
+    def permute_and_experts(self, l, T):
+        """dispatch + expert forward of layer l from x_l and its routing decision (also the
+        recompute step of backward)."""
+        c, s = self.ctx, self.slot(l)
         c.dispatch(self.x[l], T, self.idx[l], self.m, self.offsets[l], self.row_of[l], self.token_of[l],
-                   self.tile_expert[l], self.Xp[l])
-        c.expert_fwd(self.Xp[l], self.offsets[l], self.tile_expert[l], self.W_gu, self.W_down,
-                     self.base(l), self.m, self.GU[l], self.A[l], self.Yp[l])
-        c.combine(self.Yp[l], self.row_of[l], self.gate[l], T, self.x[l], self.x[l + 1])
+                   self.tile_expert[l], self.Xp[s])
+        c.expert_fwd(self.Xp[s], self.offsets[l], self.tile_expert[l], self.W_gu, self.W_down,
+                     self.base(l), self.m, self.GU[s], self.A[s], self.Yp[s])
 
     def forward(self, x0=None, T=None):
         T = self.T if T is None else T
@@ -125,7 +141,8 @@ class UniPoolStack:
         c = self.ctx
         if self.private:
             for l in range(self.L):
-                c.pool_aux_loss(self.counts[l], self.score_sum[l], 1, self.m, T, self.alpha, None,
+                c.pool_aux_loss(self.counts[l], self.score_sum[l], 1, self.m, T, self.alpha,
+                                None if fbar_prev is None else fbar_prev[l],
                                 self.loss[l:l + 1], self.coef[l], self.fbar[l])
         else:
             c.pool_aux_loss(self.counts, self.score_sum, self.L, self.m, T, self.alpha, fbar_prev,
@@ -139,9 +156,12 @@ class UniPoolStack:
         T = self.T if T is None else T
         c = self.ctx
         s = l if self.deferred_wgrad else 0
+        a = self.slot(l)
+        if self.recompute:
+            self.permute_and_experts(l, T)
         flags = B.BWD_SKIP_WGRAD if self.deferred_wgrad else (B.WGRAD_OVERWRITE if overwrite else 0)
         c.expert_bwd(dx_next, T, self.row_of[l], self.gate[l], self.token_of[l], self.offsets[l],
-                     self.tile_expert[l], self.Xp[l], self.GU[l], self.A[l], self.Yp[l], self.W_gu,
+                     self.tile_expert[l], self.Xp[a], self.GU[a], self.A[a], self.Yp[a], self.W_gu,
                      self.W_down, self.base(l), self.m, dx_next, self.dYp[s], self.dGU[s], dx_out,
                      self.dgate, self.dW_gu, self.dW_down, flags)
         coef = None
@@ -174,6 +194,26 @@ class UniPoolStack:
         if not accumulate:
             self.zero_router_grad()
         return self.backward(upstream, T, accumulate=accumulate)
+
+    def accumulate_microbatches(self, batches, fbar0=None, T=None):
+        """One optimizer step's worth of the path (App. D, App. G): every micro-batch (x0, upstream)
+        runs forward, balance loss and backward; all of them add into the same gradient buffers (the
+        first one overwrites them), and the balance loss of a micro-batch uses the token fractions
+        f-bar of the PREVIOUS micro-batch - ``fbar0`` for the first (default: the f-bar this stack saw
+        last, or uniform 1/m).  Returns the per-micro-batch losses (device tensors)."""
+        if fbar0 is not None:
+            self.fbar_lag = fbar0.to(self.device, torch.float32).reshape(self.fbar.shape).clone()
+        elif self.fbar_lag is None:
+            self.fbar_lag = torch.full_like(self.fbar, 1.0 / self.m)
+        losses = []
+        self.zero_router_grad()
+        for i, (x0, upstream) in enumerate(batches):
+            self.forward(x0, T)
+            self.aux_loss(T, fbar_prev=self.fbar_lag if self.private else self.fbar_lag[0])
+            losses.append(self.loss.clone())
+            self.fbar_lag.copy_(self.fbar)             # updated after all layers finished forward, no gradient
+            self.backward(upstream, T, accumulate=i > 0)
+        return losses
 
     def capture_step(self, x0=None, upstream=None, accumulate=True):
         """Records one whole step (the library calls of ``step`` with these tensors) into a CUDA graph

@@ -333,6 +333,78 @@ def test_one_step_behind_fbar():
     st.close()
 
 
+def test_microbatches_accumulate_with_one_step_behind_fbar():
+    """App. G: three micro-batches add into the same gradient buffers; the balance loss of each uses
+    the token fractions of the one before (uniform for the first).  Against the float64 oracle run
+    micro-batch by micro-batch with the same lagged f-bar."""
+    import torch
+    cfg = synth.CONFIGS["tiny_fp32"]
+    L, T, k, M = cfg["L"], cfg["T"], cfg["k"], cfg["M"]
+    base = synth.make_inputs(cfg, seed=0)
+    pool, routers = oracle_params(base, L)
+    st = build_stack(cfg, base)
+    batches, idxs = [], []
+    for i in range(3):
+        inp = synth.make_inputs(cfg, seed=20 + i)
+        x0, up = torch.from_numpy(inp["x0"]).cuda(), torch.from_numpy(inp["upstream"]).cuda()
+        st.forward(x0)
+        torch.cuda.synchronize()
+        idxs.append([to_np(st.idx[l]).copy() for l in range(L)])
+        batches.append((x0, up, inp))
+    st.dW_gu.fill_(9.0); st.dW_down.fill_(9.0)              # the first micro-batch overwrites
+    losses = st.accumulate_microbatches([(b[0], b[1]) for b in batches])
+    torch.cuda.synchronize()
+    prev = np.full(M, 1.0 / M)
+    tot_pool = O.zeros_like_pool(pool)
+    tot_wr = [0.0] * L
+    for i, (_, _, inp) in enumerate(batches):
+        res = O.stack_objective_and_grads(f64(inp["x0"]), routers, pool, k, st.c, synth.EPS, synth.ALPHA,
+                                          f64(inp["upstream"]), forced_idx=idxs[i], fbar_prev=prev)
+        assert abs(float(losses[i][0]) - res["loss_aux"]) <= 1e-5 * abs(res["loss_aux"])
+        for n in tot_pool:
+            tot_pool[n] += res["pool_grad"][n]
+        for l in range(L):
+            tot_wr[l] = tot_wr[l] + res["router_grads"][l]["dW_r"]
+        prev = O.pool_aux_loss(res["counts"], res["S"], T, k, synth.ALPHA)[1]       # this batch's f-bar
+    f = cfg["f"]
+    assert rel_max(to_np(st.dW_gu)[:, :f], tot_pool["W_gate"]) < 1e-5
+    assert rel_max(to_np(st.dW_gu)[:, f:], tot_pool["W_up"]) < 1e-5
+    assert rel_max(to_np(st.dW_down), tot_pool["W_down"]) < 1e-5
+    for l in range(L):
+        assert rel_max(to_np(st.dW_r[l]), tot_wr[l]) < 1e-5
+    assert rel_max(to_np(st.fbar_lag[0]), prev) < 1e-6
+    st.ctx.check_status()
+    st.close()
+
+
+def test_recomputed_activations_give_the_same_step():
+    """MoE-layer activation recompute: keeping only x_l and the routing state and rebuilding the
+    permuted activations in backward reproduces the step bit for bit."""
+    import torch
+    cfg = small_cfg(dtype="bf16", d=256, f=384, M=16, k=2, L=3)
+    T = 900
+    inputs = synth.make_inputs(cfg, seed=12, T=T)
+    x0 = torch.from_numpy(inputs["x0"]).cuda().bfloat16()
+    up = torch.from_numpy(inputs["upstream"]).cuda().bfloat16()
+    outs = []
+    for recompute in (False, True):
+        from paper_2605_06665_b200.stack import UniPoolStack
+        st = UniPoolStack(cfg["L"], cfg["d"], cfg["f"], cfg["M"], cfg["k"], T, "bf16", 0, c=2.5, eps=synth.EPS,
+                          alpha=synth.ALPHA, recompute=recompute)
+        st.load(inputs["pool"], inputs["routers"])
+        assert st.Xp.shape[0] == (1 if recompute else cfg["L"])
+        st.zero_grad()
+        dx0 = st.step(x0, up).clone()
+        torch.cuda.synchronize()
+        st.ctx.check_status()
+        outs.append([t.clone() for t in (st.x[cfg["L"]], dx0, st.dW_gu, st.dW_down, st.dW_r)])
+        st.close()
+    for a, b in zip(outs[0][:4], outs[1][:4]):
+        assert torch.equal(a, b)
+    assert rel_max(to_np(outs[1][4]), to_np(outs[0][4])) < 1e-5     # router dW: split-K add-reduce, order may differ
+    assert outs[0][2].abs().max() > 0
+
+
 def test_calibrate_c_on_device():
     from oracle import norm_router_c
     cfg = small_cfg()
