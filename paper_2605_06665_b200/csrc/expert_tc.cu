@@ -92,7 +92,11 @@ template <int MODE>
 __device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int tile, int n_nt, int n_mt) {
   TileCoord c;
   if constexpr (Traits<MODE>::kRowTiles) {
-    c.mt = tile / n_nt;
+    // A kernel that consumes what the previous launch produced in ascending row order (the down
+    // projection reads A, the second dgrad reads dGU) walks the rows downwards: the rows written
+    // last are the ones still in L2.
+    constexpr bool kDescending = MODE == kFwd2 || MODE == kDgrad2;
+    c.mt = kDescending ? n_mt - 1 - tile / n_nt : tile / n_nt;
     c.nt = tile % n_nt;
     c.e = p.tile_expert ? p.tile_expert[c.mt] : 0;
     c.kblocks = p.Kdim / BK;
