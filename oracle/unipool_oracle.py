@@ -328,12 +328,15 @@ def zeros_like_pool(pool):
 
 
 def stack_objective_and_grads(x0, routers, pool, k, c, eps, alpha, upstream, views=None,
-                              forced_idx=None, fbar_prev=None, n_view=None):
+                              forced_idx=None, fbar_prev=None, n_view=None, aux_groups=None):
     """J = sum(upstream * x_L) + balance loss, and dJ/d(everything).
 
     UniPool (views None): balance loss = Eq. 5 over all L layers.  Layer-private
     layout (views given, each layer owning ``n_view`` experts): balance loss =
-    sum_l Eq. 3.  Routing decisions and f-bar are constants of the derivative.
+    sum_l Eq. 3.  Sharing scope G (Sec. 5.3 ablation: G pools over depth): ``aux_groups`` lists the
+    layers of every group; each group is a pool of its own, so its balance loss is Eq. 5 over the
+    group's layers and experts (G = L gives sum_l Eq. 3, G = 1 gives Eq. 5).
+    Routing decisions and f-bar are constants of the derivative.
     Returns dict(J, loss_aux, caches, pool_grad, router_grads [L], dx0).
     """
     L = len(routers)
@@ -341,7 +344,15 @@ def stack_objective_and_grads(x0, routers, pool, k, c, eps, alpha, upstream, vie
     caches = stack_forward(x0, routers, pool, k, c, eps, views, forced_idx)
     counts = np.stack([cch["counts"] for cch in caches])
     S = np.stack([cch["S"] for cch in caches])
-    if views is None:
+    if aux_groups is not None:
+        loss_aux = 0.0
+        coefs = [None] * L
+        for layers in aux_groups:
+            lo, _, co = pool_aux_loss(counts[layers], S[layers], T, k, alpha)
+            loss_aux += lo
+            for l in layers:
+                coefs[l] = co
+    elif views is None:
         loss_aux, fbar, coef = pool_aux_loss(counts, S, T, k, alpha, fbar_prev)
         coefs = [coef] * L
     else:

@@ -8,7 +8,11 @@ CUDA kernel of the library.
 
 Layer l computes x_{l+1} = x_l + sum_{i in top-k} g_{l,i}(x_l) e_i(x_l)  (Eq. 2),
 all layers sharing one pool of experts; with ``private = E`` layer l instead
-owns pool experts [E*l, E*(l+1)) (the layer-private layout of Eq. 1) and the
+owns pool experts [E*l, E*(l+1)) (the layer-private layout of Eq. 1); with
+``groups = G`` (sharing scope of the ablation in Sec. 5.3) the L layers form G
+consecutive groups of L/G layers, group g sharing pool experts [g*M/G, (g+1)*M/G)
+with its own balance loss (Eq. 5 over the group's layers; G = 1 is UniPool, G = L
+the private layout).  In the private layout the
 balance loss is the per-layer loss of Eq. 3 summed over layers.
 """
 from __future__ import annotations
@@ -21,17 +25,22 @@ from . import binding as B
 
 class UniPoolStack:
     def __init__(self, L, d, f, M, k, T, dtype="bf16", private=0, c=1.0, eps=1e-6, alpha=1e-2,
-                 device="cuda", deferred_wgrad=False, recompute=False):
+                 device="cuda", deferred_wgrad=False, recompute=False, groups=None):
         self.L, self.d, self.f, self.M, self.k, self.T = L, d, f, M, k, T
+        if groups is None:
+            groups = L if private else 1
+        if L % groups or M % groups or (private and (groups != L or private * L != M)):
+            raise ValueError("layers and pool experts must split evenly into the sharing groups")
+        self.G, self.Lg = groups, L // groups              # sharing groups over depth, layers per group
         self.private = private
-        self.m = private if private else M                 # experts one router scores
+        self.m = M // groups                               # experts one router scores
         self.alpha = alpha
         self.c, self.eps = c, eps
         # recompute: keep only x_l and the routing state of a layer; its permuted activations are
         # rebuilt in backward (MoE-layer activation recompute, App. D), so the weight gradient is
         # taken layer by layer
         self.recompute = recompute
-        self.deferred_wgrad = deferred_wgrad and not private and not recompute
+        self.deferred_wgrad = deferred_wgrad and self.Lg > 1 and not recompute
         self.device = torch.device(device)
         self.tdtype = torch.bfloat16 if dtype == "bf16" else torch.float32
         self.cfg = B.make_config(d, f, M, k, L, T, B.BF16 if dtype == "bf16" else B.FP32, eps, c)
@@ -75,7 +84,7 @@ class UniPoolStack:
         self.dx = e(2, T, d)                               # ping-pong dx_{l+1} -> dx_l
         self.dgate = e(T, k, dtype=f32)
         # balance loss
-        n_aux = L if private else 1
+        n_aux = groups                                     # one balance loss per sharing group
         self.loss = torch.zeros(n_aux, dtype=f32, device=dev)
         self.coef = e(n_aux, self.m, dtype=f32)
         self.fbar = e(n_aux, self.m, dtype=f32)
@@ -97,7 +106,7 @@ class UniPoolStack:
         torch.cuda.synchronize(self.device)
 
     def base(self, l):
-        return self.private * l if self.private else 0
+        return (l // self.Lg) * self.m
 
     def slot(self, l):
         """Index of layer l's permuted activations (one shared slot when they are recomputed)."""
@@ -139,14 +148,13 @@ class UniPoolStack:
     def aux_loss(self, T=None, fbar_prev=None):
         T = self.T if T is None else T
         c = self.ctx
-        if self.private:
-            for l in range(self.L):
-                c.pool_aux_loss(self.counts[l], self.score_sum[l], 1, self.m, T, self.alpha,
-                                None if fbar_prev is None else fbar_prev[l],
-                                self.loss[l:l + 1], self.coef[l], self.fbar[l])
-        else:
-            c.pool_aux_loss(self.counts, self.score_sum, self.L, self.m, T, self.alpha, fbar_prev,
-                            self.loss, self.coef[0], self.fbar[0])
+        if fbar_prev is not None and fbar_prev.dim() == 1:
+            fbar_prev = fbar_prev.reshape(1, -1)
+        for g in range(self.G):
+            l0 = g * self.Lg
+            c.pool_aux_loss(self.counts[l0:l0 + self.Lg], self.score_sum[l0:l0 + self.Lg], self.Lg, self.m, T,
+                            self.alpha, None if fbar_prev is None else fbar_prev[g],
+                            self.loss[g:g + 1], self.coef[g], self.fbar[g])
         return self.loss
 
     # ------------------------------------------------------------------ backward
@@ -166,7 +174,7 @@ class UniPoolStack:
                      self.dgate, self.dW_gu, self.dW_down, flags)
         coef = None
         if with_aux:
-            coef = self.coef[l] if self.private else self.coef[0]
+            coef = self.coef[l // self.Lg]
         c.route_bwd(self.x[l], T, self.W_r[l], self.sigma[l], self.m, self.znorm[l], self.z[l],
                     self.idx[l], self.dgate, coef, dx_out, self.dW_r[l], self.dsigma[l:l + 1])
 
@@ -179,12 +187,15 @@ class UniPoolStack:
         if upstream is not None:
             self.dx[cur, :T].copy_(upstream, non_blocking=True)
         for l in reversed(range(self.L)):
-            first = (not accumulate) and (bool(self.private) or l == self.L - 1)
+            first = (not accumulate) and l % self.Lg == self.Lg - 1     # first contribution to its group's experts
             self.backward_layer(l, self.dx[cur], self.dx[1 - cur], T, with_aux, overwrite=first)
             cur = 1 - cur
         if self.deferred_wgrad:
-            self.ctx.pool_wgrad(self.L, self.cap, self.offsets, self.Xp, self.A, self.dYp, self.dGU,
-                                0, self.m, self.dW_gu, self.dW_down, 0 if accumulate else B.WGRAD_OVERWRITE)
+            for g in range(self.G):                        # one pass per sharing group over its layers
+                l0 = g * self.Lg
+                self.ctx.pool_wgrad(self.Lg, self.cap, self.offsets[l0:], self.Xp[l0:], self.A[l0:], self.dYp[l0:],
+                                    self.dGU[l0:], g * self.m, self.m, self.dW_gu, self.dW_down,
+                                    0 if accumulate else B.WGRAD_OVERWRITE)
         return self.dx[cur]
 
     def step(self, x0=None, upstream=None, T=None, accumulate=True):
@@ -209,7 +220,7 @@ class UniPoolStack:
         self.zero_router_grad()
         for i, (x0, upstream) in enumerate(batches):
             self.forward(x0, T)
-            self.aux_loss(T, fbar_prev=self.fbar_lag if self.private else self.fbar_lag[0])
+            self.aux_loss(T, fbar_prev=self.fbar_lag)
             losses.append(self.loss.clone())
             self.fbar_lag.copy_(self.fbar)             # updated after all layers finished forward, no gradient
             self.backward(upstream, T, accumulate=i > 0)

@@ -65,12 +65,17 @@ def _normal(seed, tag, layer, shape, std, bf16):
 
 
 def router_width(cfg):
-    """Number of experts one router scores: M (shared pool) or the private count."""
+    """Number of experts one router scores: M (shared pool), the private count, or M / G when the
+    layers form ``groups`` = G sharing groups over depth."""
+    if cfg.get("groups"):
+        return cfg["M"] // cfg["groups"]
     return cfg["private"] if cfg["private"] else cfg["M"]
 
 
 def expert_base(cfg, layer):
     """First pool expert visible to ``layer``'s router."""
+    if cfg.get("groups"):
+        return (layer // (cfg["L"] // cfg["groups"])) * (cfg["M"] // cfg["groups"])
     return cfg["private"] * layer if cfg["private"] else 0
 
 

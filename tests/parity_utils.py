@@ -86,7 +86,7 @@ def build_stack(cfg, inputs, T=None, L=None, deferred_wgrad=False, c=None):
     m = synth.router_width(cfg)
     c = calib_c(m, cfg["k"]) if c is None else c
     st = UniPoolStack(L, cfg["d"], cfg["f"], cfg["M"], cfg["k"], T, cfg["dtype"], cfg["private"], c=c,
-                      eps=synth.EPS, alpha=synth.ALPHA, deferred_wgrad=deferred_wgrad)
+                      eps=synth.EPS, alpha=synth.ALPHA, deferred_wgrad=deferred_wgrad, groups=cfg.get("groups"))
     st.load(inputs["pool"], inputs["routers"][:L])
     return st
 

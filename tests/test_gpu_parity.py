@@ -405,6 +405,52 @@ def test_recomputed_activations_give_the_same_step():
     assert outs[0][2].abs().max() > 0
 
 
+@pytest.mark.parametrize("dtype,deferred", [("fp32", False), ("fp32", True), ("bf16", True)])
+def test_sharing_scope_groups(dtype, deferred):
+    """G = 2 sharing groups over L = 4 layers (the ablation's intermediate sharing scope): layers
+    {0,1} share pool experts 0..7, layers {2,3} experts 8..15, each group with its own Eq. 5 loss.
+    Whole step against the float64 oracle (forced to the GPU's routing)."""
+    import torch
+    cfg = small_cfg(dtype=dtype, d=128, f=192, M=16, k=2, L=4, groups=2)
+    T = 400
+    inputs = synth.make_inputs(cfg, seed=14, T=T)
+    st = build_stack(cfg, inputs, T=T, deferred_wgrad=deferred)
+    assert st.m == 8 and st.G == 2 and st.deferred_wgrad == deferred
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    x0 = torch.from_numpy(inputs["x0"]).cuda().to(tdt)
+    up = torch.from_numpy(inputs["upstream"]).cuda().to(tdt)
+    st.dW_gu.fill_(4.0); st.dW_down.fill_(4.0)
+    st.step(x0, up, accumulate=False)
+    torch.cuda.synchronize()
+    st.ctx.check_status()
+    pool, routers = oracle_params(inputs, 4)
+    views = [synth.expert_base(cfg, l) for l in range(4)]
+    assert views == [0, 0, 8, 8]
+    idx = [to_np(st.idx[l]) for l in range(4)]
+    if dtype == "fp32":
+        res = O.stack_objective_and_grads(f64(inputs["x0"]), routers, pool, 2, st.c, synth.EPS, synth.ALPHA,
+                                          f64(inputs["upstream"]), views, forced_idx=idx, aux_groups=[[0, 1], [2, 3]])
+        tol = 1e-5
+        assert rel_max(to_np(st.x[4]), res["caches"][-1]["x_next"]) < tol
+        assert abs(float(st.loss.sum()) - res["loss_aux"]) <= 1e-5 * abs(res["loss_aux"])
+        f = cfg["f"]
+        assert rel_max(to_np(st.dW_gu)[:, :f], res["pool_grad"]["W_gate"]) < tol
+        assert rel_max(to_np(st.dW_down), res["pool_grad"]["W_down"]) < tol
+        for l in range(4):
+            assert rel_max(to_np(st.dW_r[l]), res["router_grads"][l]["dW_r"]) < tol
+    else:
+        # bf16: the grouped one-pass weight gradient must equal the per-layer accumulation
+        ref = build_stack(cfg, inputs, T=T, deferred_wgrad=False)
+        ref.zero_grad()
+        ref.step(x0, up)
+        torch.cuda.synchronize()
+        assert rel_max(to_np(st.dW_gu), to_np(ref.dW_gu)) < 1e-5
+        assert rel_max(to_np(st.dW_down), to_np(ref.dW_down)) < 1e-5
+        assert torch.equal(st.x[4], ref.x[4])
+        ref.close()
+    st.close()
+
+
 def test_calibrate_c_on_device():
     from oracle import norm_router_c
     cfg = small_cfg()

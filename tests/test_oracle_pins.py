@@ -296,6 +296,52 @@ def test_backward_matches_central_finite_differences(private, bias):
     assert checked >= 9
 
 
+def test_sharing_scope_groups_interpolate_between_pool_and_private():
+    """G pools over depth: G = 1 is the shared pool (Eq. 5), G = L the layer-private layout
+    (sum of Eq. 3), and for G = 2 the gradient of the grouped objective matches finite differences."""
+    pool, routers, x0, up, _ = tiny_problem(seed=5, L=4, M=6, d=8, f=5, k=2, T=10)
+    k, c, eps, alpha = 2, 1.9, 1e-6, 0.5
+    one = O.stack_objective_and_grads(x0, routers, pool, k, c, eps, alpha, up)
+    g1 = O.stack_objective_and_grads(x0, routers, pool, k, c, eps, alpha, up, views=[0] * 4,
+                                     aux_groups=[[0, 1, 2, 3]])
+    assert g1["J"] == pytest.approx(one["J"], rel=1e-14)
+    np.testing.assert_allclose(g1["pool_grad"]["W_up"], one["pool_grad"]["W_up"], rtol=1e-12, atol=1e-14)
+    # G = L with 4 private experts of 6... use a pool of 8 = 4 layers x 2 experts
+    pool8, routers8, x0, up, views = tiny_problem(seed=6, L=4, M=8, d=8, f=5, k=2, T=10, private=2)
+    priv = O.stack_objective_and_grads(x0, routers8, pool8, k, c, eps, alpha, up, views, n_view=2)
+    gL = O.stack_objective_and_grads(x0, routers8, pool8, k, c, eps, alpha, up, views,
+                                     aux_groups=[[0], [1], [2], [3]])
+    assert gL["J"] == pytest.approx(priv["J"], rel=1e-14)
+    np.testing.assert_allclose(gL["router_grads"][2]["dW_r"], priv["router_grads"][2]["dW_r"], rtol=1e-12)
+    # G = 2: layers {0,1} share experts 0..3, layers {2,3} share experts 4..7; routers score 4 experts
+    rng = np.random.default_rng(3)
+    routers2 = [dict(W_r=rng.normal(0, 0.5, (4, 8)), sigma=1.0 + 0.1 * l, bias=None) for l in range(4)]
+    views2, groups2 = [0, 0, 4, 4], [[0, 1], [2, 3]]
+    res = O.stack_objective_and_grads(x0, routers2, pool8, k, c, eps, alpha, up, views2, aux_groups=groups2)
+    base_idx = [cc["idx"] for cc in res["caches"]]
+
+    def J():
+        r = O.stack_objective_and_grads(x0, routers2, pool8, k, c, eps, alpha, up, views2, aux_groups=groups2)
+        for a, b in zip(r["caches"], base_idx):
+            assert (a["idx"] == b).all()
+        return r["J"]
+
+    def fd(arr, pos, h=1e-6):
+        old = arr[pos]
+        arr[pos] = old + h; jp = J()
+        arr[pos] = old - h; jm = J()
+        arr[pos] = old
+        return (jp - jm) / (2 * h)
+
+    used = np.unique(np.concatenate([views2[l] + cc["idx"].reshape(-1) for l, cc in enumerate(res["caches"])]))
+    for e in used[:5]:
+        pos = (int(e), int(rng.integers(0, 5)), int(rng.integers(0, 8)))
+        assert fd(pool8["W_gate"], pos) == pytest.approx(res["pool_grad"]["W_gate"][pos], rel=2e-5, abs=1e-8)
+    for l in range(4):
+        pos = (int(rng.integers(0, 4)), int(rng.integers(0, 8)))
+        assert fd(routers2[l]["W_r"], pos) == pytest.approx(res["router_grads"][l]["dW_r"][pos], rel=2e-5, abs=1e-8)
+
+
 def test_shared_pool_gradient_is_the_sum_over_layers():
     """Each shared expert accumulates gradient from all L layers (Sec. 3): running the
     layers' backward passes one at a time into separate buffers and adding them gives
