@@ -240,6 +240,16 @@ int unipool_route_bwd(unipool_ctx* ctx, const void* x, int32_t T, const float* W
                       const int32_t* idx, const float* dgate, const float* dscore_coef,
                       void* dx, float* dW_r, float* dsigma, unipool_stream stream);
 
+/* Distinct-expert accounting (App. E): U(x) = |{ e_l(x) : l = 1..L }|, the number of different pool
+ * experts a token selects over all layers (the paper states it for top-1; with top-k every selected
+ * expert of every layer counts).  With the shared pool 1 <= U <= min(M, L k); with private experts
+ * (expert_base[l] = first pool expert of layer l) U = L k.
+ * in : idx [L,T,k] int32 (the routers' indices of all layers, stacked); expert_base [L] int32 or NULL
+ *      (= 0 for every layer).  Ids outside the pool are ignored.
+ * out: unique [T] int32; total (device uint64) = sum over tokens of U(x) (mean = total / T). */
+int unipool_unique_experts(unipool_ctx* ctx, const int32_t* idx, const int32_t* expert_base, int32_t L,
+                           int32_t T, int32_t* unique, uint64_t* total, unipool_stream stream);
+
 /* Monte-Carlo estimate of the NormRouter constant c (Alg. 1):
  *   c = E[ 1 / ||top-k(ReLU(x/||x||_2))||_2 ],  x ~ N(0, I_E),
  * over n_samples draws of a counter-based generator seeded by `seed`; draws

@@ -323,6 +323,23 @@ def layer_backward(cache, router, pool, k, c, eps, dx_next, coef, pool_grad, exp
                 dx_expert=dx_e, dx_router=rb["dx"])
 
 
+def unique_experts(idx_layers, views=None):
+    """App. E: U(x) = |{ e_l(x) : l = 1..L }| per token - the number of distinct pool experts the
+    token selects over all layers (every one of the k picks of a layer counts).  ``idx_layers`` is a
+    list of [T,k] index arrays, ``views[l]`` the first pool expert of layer l (None: shared pool)."""
+    L = len(idx_layers)
+    T = idx_layers[0].shape[0]
+    out = np.zeros(T, dtype=np.int64)
+    for t in range(T):
+        seen = set()
+        for l in range(L):
+            base = 0 if views is None else views[l]
+            for e in idx_layers[l][t]:
+                seen.add(base + int(e))
+        out[t] = len(seen)
+    return out
+
+
 def zeros_like_pool(pool):
     return {name: np.zeros_like(w) for name, w in pool.items()}
 

@@ -24,6 +24,7 @@ EXPORTS = (
     "unipool_expert_fwd", "unipool_combine", "unipool_expert_bwd", "unipool_pool_wgrad",
     "unipool_pool_aux_loss", "unipool_route_bwd", "unipool_calibrate_c",
     "unipool_profile_enable", "unipool_profile_read", "unipool_dispatch_static",
+    "unipool_unique_experts",
 )
 
 PHASES = (
@@ -93,6 +94,8 @@ def lib():
     L.unipool_pool_aux_loss.argtypes = [vp, vp, vp, i32, i32, i32, f32, vp, vp, vp, vp, vp]
     L.unipool_route_bwd.restype = ctypes.c_int
     L.unipool_route_bwd.argtypes = [vp, vp, i32, vp, f32, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    L.unipool_unique_experts.restype = ctypes.c_int
+    L.unipool_unique_experts.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp]
     L.unipool_calibrate_c.restype = ctypes.c_int
     L.unipool_calibrate_c.argtypes = [vp, i32, i32, i32, ctypes.c_uint64, ctypes.POINTER(f32), vp]
     L.unipool_profile_enable.restype = ctypes.c_int
@@ -209,6 +212,10 @@ class Context:
         _check(lib().unipool_route_bwd(self.handle, _p(x), T, _p(W_r), sigma, n_experts, _p(znorm),
                                        _p(z_saved), _p(idx), _p(dgate), _p(dscore_coef), _p(dx), _p(dW_r),
                                        _p(dsigma), _stream()))
+
+    def unique_experts(self, idx, expert_base, L, T, unique, total):
+        _check(lib().unipool_unique_experts(self.handle, _p(idx), _p(expert_base), L, T, _p(unique), _p(total),
+                                            _stream()))
 
     def profile_enable(self, on):
         _check(lib().unipool_profile_enable(self.handle, 1 if on else 0))

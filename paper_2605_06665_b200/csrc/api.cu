@@ -315,6 +315,14 @@ int unipool_route_bwd(unipool_ctx* ctx, const void* x, int32_t T, const float* W
                           dscore_coef, dx, dW_r, dsigma, static_cast<cudaStream_t>(stream));
 }
 
+int unipool_unique_experts(unipool_ctx* ctx, const int32_t* idx, const int32_t* expert_base, int32_t L,
+                           int32_t T, int32_t* unique, uint64_t* total, unipool_stream stream) {
+  CHECK_CTX(ctx); CHECK_T(ctx, T); CHECK_PTR(idx); CHECK_PTR(unique); CHECK_PTR(total);
+  UP_REQUIRE(L >= 1, UNIPOOL_ERR_INVALID_ARG, "L must be >= 1");
+  return unique_experts_launch(ctx, idx, expert_base, L, T, unique, reinterpret_cast<unsigned long long*>(total),
+                               static_cast<cudaStream_t>(stream));
+}
+
 int unipool_calibrate_c(unipool_ctx* ctx, int32_t n_experts, int32_t top_k, int32_t n_samples,
                         uint64_t seed, float* c_out, unipool_stream stream) {
   CHECK_CTX(ctx); CHECK_PTR(c_out);

@@ -42,6 +42,48 @@ int aux_launch(unipool_ctx* ctx, const int32_t* counts, const float* S, int L, i
   return UNIPOOL_OK;
 }
 
+// ---------------------------------------------------------------- distinct-expert accounting (App. E)
+// U(x) = |{ pool experts token x selects in any layer }|; one thread per token keeps a bit set of
+// the M <= 512 pool experts.  idx is [L, T, k] (router-local ids), expert_base[l] maps layer l's ids
+// into the pool (0 everywhere for the shared pool).
+__global__ void __launch_bounds__(256)
+unique_experts_kernel(const int32_t* __restrict__ idx, const int32_t* __restrict__ expert_base, int L, int T,
+                      int k, int M, int32_t* __restrict__ unique, unsigned long long* __restrict__ total) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  int u = 0;
+  if (t < T) {
+    uint32_t bits[UNIPOOL_MAX_EXPERTS / 32];
+#pragma unroll
+    for (int w = 0; w < UNIPOOL_MAX_EXPERTS / 32; ++w) bits[w] = 0u;
+    for (int l = 0; l < L; ++l) {
+      const int base = expert_base ? expert_base[l] : 0;
+      for (int j = 0; j < k; ++j) {
+        const int e = base + idx[((int64_t)l * T + t) * k + j];
+        if (e < 0 || e >= M) continue;               // dropped assignment
+#pragma unroll
+        for (int w = 0; w < UNIPOOL_MAX_EXPERTS / 32; ++w)
+          if (w == (e >> 5)) bits[w] |= 1u << (e & 31);
+      }
+    }
+#pragma unroll
+    for (int w = 0; w < UNIPOOL_MAX_EXPERTS / 32; ++w) u += __popc(bits[w]);
+    unique[t] = u;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) u += __shfl_xor_sync(0xffffffffu, u, o);
+  if ((threadIdx.x & 31) == 0 && u) atomicAdd(total, (unsigned long long)u);
+}
+
+int unique_experts_launch(unipool_ctx* ctx, const int32_t* idx, const int32_t* expert_base, int L, int T,
+                          int32_t* unique, unsigned long long* total, cudaStream_t s) {
+  UP_CUDA(cudaMemsetAsync(total, 0, sizeof(unsigned long long), s));
+  if (T == 0) return UNIPOOL_OK;
+  unique_experts_kernel<<<(T + 255) / 256, 256, 0, s>>>(idx, expert_base, L, T, ctx->cfg.top_k, ctx->cfg.pool_size,
+                                                       unique, total);
+  UP_LAUNCH_CHECK();
+  return UNIPOOL_OK;
+}
+
 // ---------------------------------------------------------------- Alg. 1
 // Counter-based generator: a 64-bit mix of (seed, sample, element) gives two
 // uniform 32-bit words, turned into one normal draw by Box-Muller.

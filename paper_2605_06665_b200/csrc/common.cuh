@@ -150,6 +150,8 @@ int unpermute_sum_launch(unipool_ctx*, const void* dXp, const int32_t* row_of, i
 int aux_launch(unipool_ctx*, const int32_t* counts, const float* S, int L, int n_experts, int T,
                float alpha, const float* fbar_prev, float* loss, float* coef, float* fbar_out,
                cudaStream_t);
+int unique_experts_launch(unipool_ctx*, const int32_t* idx, const int32_t* expert_base, int L, int T,
+                          int32_t* unique, unsigned long long* total, cudaStream_t);
 int calibrate_launch(unipool_ctx*, int n_experts, int top_k, int n_samples, uint64_t seed,
                      float* c_out, cudaStream_t);
 

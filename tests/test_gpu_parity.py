@@ -451,6 +451,29 @@ def test_sharing_scope_groups(dtype, deferred):
     st.close()
 
 
+@pytest.mark.parametrize("kw", [dict(M=8, k=2, L=4), dict(M=12, k=2, private=4, L=3), dict(M=40, k=8, d=64, f=64, L=2)])
+def test_unique_experts_per_token(kw):
+    """App. E's U(x) over the routing decisions of a real forward pass, bit-exact against the oracle."""
+    import torch
+    cfg = small_cfg(**kw)
+    T, L = 257, cfg["L"]
+    inputs = synth.make_inputs(cfg, seed=2, T=T)
+    st = build_stack(cfg, inputs, T=T)
+    st.forward(torch.from_numpy(inputs["x0"]).cuda())
+    views = [synth.expert_base(cfg, l) for l in range(L)]
+    base = torch.tensor(views, dtype=torch.int32, device="cuda") if cfg["private"] else None
+    unique = torch.full((T,), -1, dtype=torch.int32, device="cuda")
+    total = torch.full((1,), 77, dtype=torch.int64, device="cuda")
+    st.ctx.unique_experts(st.idx, base, L, T, unique, total)
+    torch.cuda.synchronize()
+    ref = O.unique_experts([to_np(st.idx[l]) for l in range(L)], views if cfg["private"] else None)
+    assert (to_np(unique) == ref).all()
+    assert int(total[0]) == int(ref.sum())
+    if cfg["private"]:
+        assert (ref == L * cfg["k"]).all()
+    st.close()
+
+
 def test_calibrate_c_on_device():
     from oracle import norm_router_c
     cfg = small_cfg()

@@ -342,6 +342,26 @@ def test_sharing_scope_groups_interpolate_between_pool_and_private():
         assert fd(routers2[l]["W_r"], pos) == pytest.approx(res["router_grads"][l]["dW_r"][pos], rel=2e-5, abs=1e-8)
 
 
+def test_unique_expert_accounting():
+    """App. E: private experts give U = L exactly for top-1 (L k for top-k); a shared pool gives
+    1 <= U <= min(M, L k); a hand case; and U equals the row-wise count of a dense indicator matrix."""
+    rng = np.random.default_rng(0)
+    L, T, k, M = 5, 40, 1, 7
+    idx = [rng.integers(0, 3, (T, k)).astype(np.int32) for _ in range(L)]
+    assert (O.unique_experts(idx, views=[3 * l for l in range(L)]) == L).all()        # vanilla: exactly L
+    U = O.unique_experts(idx)
+    assert U.min() >= 1 and U.max() <= 3
+    hand = [np.array([[0, 1]]), np.array([[1, 2]]), np.array([[0, 2]])]                   # top-2, 3 layers
+    assert O.unique_experts(hand)[0] == 3
+    assert O.unique_experts(hand, views=[0, 3, 6])[0] == 6
+    idx2 = [np.stack([rng.permutation(M)[:2] for _ in range(T)]).astype(np.int32) for _ in range(L)]
+    dense = np.zeros((T, M), bool)
+    for a in idx2:
+        for j in range(2):
+            dense[np.arange(T), a[:, j]] = True
+    assert (O.unique_experts(idx2) == dense.sum(axis=1)).all()
+
+
 def test_shared_pool_gradient_is_the_sum_over_layers():
     """Each shared expert accumulates gradient from all L layers (Sec. 3): running the
     layers' backward passes one at a time into separate buffers and adding them gives
