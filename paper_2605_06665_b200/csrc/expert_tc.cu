@@ -586,6 +586,8 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
 // even CTA issues the MMAs; every TMA load counts its bytes on the even CTA's mbarrier (plain
 // loads, no multicast); tcgen05.commit arrives on the stage / accumulator barriers of both CTAs.
 constexpr int kPairStages = 6;
+constexpr uint32_t kPairSmemTotal = kSmemTotal + UNIPOOL_MAX_EXPERTS * sizeof(uint16_t);   // + the experts' order
+static_assert(kPairSmemTotal <= 227 * 1024, "shared-memory budget");
 constexpr uint32_t kPairHalfBytes = 128 * BK * 2;            // 128 (M or N) x 64 (K) bf16
 constexpr uint32_t kPairStageBytes = 2 * kPairHalfBytes;
 static_assert(kPairStages * kPairStageBytes + kEpiWarps * 8192 == kBarOffset, "shared-memory budget");
@@ -638,6 +640,24 @@ wgrad_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   const int per_e = n_mt * n_nt;
   const int total = p.n_experts * per_e;
 
+  // Ragged groups: the contraction length of a tile is its expert's row count over all layers.  The
+  // experts are taken in order of decreasing length (ties by index), so that the round-robin over the
+  // CTA pairs deals out tiles of similar size in every round and the long ones first.
+  uint16_t* order = reinterpret_cast<uint16_t*>(smem + kBarOffset + 512);   // [n_experts] i-th longest expert
+  int* kb_of = reinterpret_cast<int*>(smem + kPairStages * kPairStageBytes);  // scratch in the (still idle) staging tiles
+  for (int e = threadIdx.x; e < p.n_experts; e += blockDim.x) kb_of[e] = wgrad_kblocks(p, e);
+  __syncthreads();
+  for (int e = threadIdx.x; e < p.n_experts; e += blockDim.x) {
+    const int mine = kb_of[e];
+    int rank_e = 0;
+    for (int o = 0; o < p.n_experts; ++o) {
+      const int other = kb_of[o];
+      rank_e += (other > mine || (other == mine && o < e)) ? 1 : 0;
+    }
+    order[rank_e] = (uint16_t)e;
+  }
+  __syncthreads();                                                           // kb_of is dead from here on
+
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer (one in each CTA)
     if (lane == 0) {
@@ -645,7 +665,7 @@ wgrad_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       uint32_t phase = 0;
       bool ok = true;
       for (int tile = pair; tile < total && ok; tile += n_pairs) {
-        const int e = tile / per_e, rem = tile % per_e, mt = rem / n_nt, nt = rem % n_nt;
+        const int e = order[tile / per_e], rem = tile % per_e, mt = rem / n_nt, nt = rem % n_nt;
         const int kblocks = wgrad_kblocks(p, e);
         int layer = 0, r = p.offsets[e], r_end = p.offsets[e + 1];
         for (int kb = 0; kb < kblocks; ++kb) {
@@ -682,7 +702,7 @@ wgrad_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       int local = 0;
       bool ok = true;
       for (int tile = pair; tile < total && ok; tile += n_pairs) {
-        const int kblocks = wgrad_kblocks(p, tile / per_e);
+        const int kblocks = wgrad_kblocks(p, order[tile / per_e]);
         if (kblocks == 0) continue;
         const int acc = local & 1;
         const uint32_t acc_phase = (local >> 1) & 1;
@@ -711,7 +731,7 @@ wgrad_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     uint8_t* stg = smem + kPairStages * kPairStageBytes + (warp - 2) * 8192;
     int gchunk = 0, local = 0;
     for (int tile = pair; tile < total; tile += n_pairs) {
-      const int e = tile / per_e, rem = tile % per_e, mt = rem / n_nt, nt = rem % n_nt;
+      const int e = order[tile / per_e], rem = tile % per_e, mt = rem / n_nt, nt = rem % n_nt;
       const int m0 = mt * 256 + rank * 128 + quarter * 32;
       const int grow = (p.expert_base + e) * p.Mdim + m0;
       if (wgrad_kblocks(p, e) == 0) {
@@ -851,8 +871,8 @@ int launch_wgrad(unipool_ctx* ctx, int phase, const CUtensorMap& tmP, const CUte
   static const bool pair = [] { const char* v = getenv("UNIPOOL_WGRAD_PAIR"); return !(v && v[0] == '0'); }();
   if (!pair || ctx->sm_count < 2) return launch<kWgrad>(ctx, phase, tmP, tmQ, tmW, tmW, p, s);
   PhaseTimer pt(ctx, phase, 1, s);
-  UP_CUDA(cudaFuncSetAttribute(wgrad_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemTotal));
-  wgrad_pair_kernel<<<ctx->sm_count / 2 * 2, kThreads, kSmemTotal, s>>>(tmP, tmQ, tmW, p);
+  UP_CUDA(cudaFuncSetAttribute(wgrad_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPairSmemTotal));
+  wgrad_pair_kernel<<<ctx->sm_count / 2 * 2, kThreads, kPairSmemTotal, s>>>(tmP, tmQ, tmW, p);
   UP_LAUNCH_CHECK();
   return UNIPOOL_OK;
 }
