@@ -56,6 +56,20 @@ def norm_router_scores(z, sigma, c, eps):
     return s.astype(z.dtype), n.astype(z.dtype)
 
 
+def softmax_router_scores(z):
+    """The conventional router the paper compares against (Sec. 4.3, first sentence; Sec. 5.1
+    "top-1 softmax routing"): s_i = exp(z_i) / sum_j exp(z_j) over the router's experts.
+
+    Returns (s [T,M], lse [T]) with lse = log sum_j exp(z_j); the largest logit is subtracted before
+    exponentiation, which changes nothing in exact arithmetic.
+    """
+    m = np.max(z, axis=-1)
+    e = np.exp(z - m[:, None])
+    tot = np.sum(e, axis=-1)
+    s = e / tot[:, None]
+    return s.astype(z.dtype), (m + np.log(tot)).astype(z.dtype)
+
+
 def top_k(s, k):
     """Indices of the k highest scores per token (Sec. 4.3, "top-k experts are
     selected based on the highest scores"), descending score, ties broken by
@@ -66,8 +80,9 @@ def top_k(s, k):
     return order[:, :k].astype(np.int32)
 
 
-def route(x, W_r, sigma, c, eps, k, bias=None, forced_idx=None):
-    """One layer's router: logits, Eq. 7 scores, top-k, gates and statistics.
+def route(x, W_r, sigma, c, eps, k, bias=None, forced_idx=None, mode="norm"):
+    """One layer's router: logits, scores (Eq. 7, or softmax with ``mode="softmax"``, where sigma, c
+    and eps play no part and ``n`` holds log-sum-exp of the logits), top-k, gates and statistics.
 
     Returns a dict with
       z [T,M], n [T], s [T,M], idx [T,k] int32, g [T,k] (g = s at idx, Eq. 2),
@@ -77,7 +92,11 @@ def route(x, W_r, sigma, c, eps, k, bias=None, forced_idx=None):
     fixed); gates are still read from s.
     """
     z = router_logits(x, W_r, bias)
-    s, n = norm_router_scores(z, sigma, c, eps)
+    if mode == "softmax":
+        s, n = softmax_router_scores(z)
+    else:
+        assert mode == "norm", mode
+        s, n = norm_router_scores(z, sigma, c, eps)
     idx = top_k(s, k) if forced_idx is None else np.asarray(forced_idx, dtype=np.int32)
     g = np.take_along_axis(s, idx.astype(np.int64), axis=1)
     M = W_r.shape[0]
@@ -165,7 +184,8 @@ def moe_layer_output(x, idx, g, pool, expert_base=0, tokens=None):
 
 def layer_forward(x, router, pool, k, c, eps, expert_base=0, forced_idx=None):
     """One residual MoE block: route, Eq. 2, x_next = x + FFN_l(x)."""
-    r = route(x, router["W_r"], router["sigma"], c, eps, k, router.get("bias"), forced_idx)
+    r = route(x, router["W_r"], router["sigma"], c, eps, k, router.get("bias"), forced_idx,
+              router.get("mode", "norm"))
     y = moe_layer_output(x, r["idx"], r["g"], pool, expert_base)
     r["y"] = y
     r["x"] = x
@@ -286,8 +306,12 @@ def expert_path_backward(x, idx, g, pool, dy, expert_base=0, pool_grad=None, tok
     return dx, dg
 
 
-def route_backward(x, W_r, sigma, c, eps, z, n, idx, dg, coef=None):
-    """Derivative of Eq. 7 followed by z = W_r x.
+def route_backward(x, W_r, sigma, c, eps, z, n, idx, dg, coef=None, mode="norm"):
+    """Derivative of the score function followed by z = W_r x.
+
+    ``mode="softmax"``: s = softmax(z), so with q_t = sum_i ds_{t,i} s_{t,i}
+        dz_{t,m} = s_{t,m} (ds_{t,m} - q_t),   dsigma = 0   (``n`` is not used).
+    ``mode="norm"`` (Eq. 7):
 
     ds_{t,i} = coef_i + sum_{j: idx_{t,j}=i} dg_{t,j}   (coef: balance-loss term)
     With u = max(z,0) and q_t = sum_i ds_{t,i} u_{t,i}:
@@ -302,6 +326,12 @@ def route_backward(x, W_r, sigma, c, eps, z, n, idx, dg, coef=None):
         ds += np.asarray(coef, dtype=z.dtype)[None, :]
     np.add.at(ds, (np.repeat(np.arange(T), idx.shape[1]), idx.reshape(-1).astype(np.int64)),
               dg.reshape(-1))
+    if mode == "softmax":
+        sm, _ = softmax_router_scores(z)
+        q = np.sum(ds * sm, axis=1)
+        dz = (sm * (ds - q[:, None])).astype(z.dtype)
+        return dict(dz=dz, dW_r=dz.T @ x, dsigma=z.dtype.type(0), dx=dz @ W_r, ds=ds)
+    assert mode == "norm", mode
     u = np.maximum(z, 0.0)
     q = np.sum(ds * u, axis=1)
     ne = n + eps
@@ -318,7 +348,7 @@ def layer_backward(cache, router, pool, k, c, eps, dx_next, coef, pool_grad, exp
     x = cache["x"]
     dx_e, dg = expert_path_backward(x, cache["idx"], cache["g"], pool, dx_next, expert_base, pool_grad)
     rb = route_backward(x, router["W_r"], router["sigma"], c, eps, cache["z"], cache["n"],
-                        cache["idx"], dg, coef)
+                        cache["idx"], dg, coef, router.get("mode", "norm"))
     return dict(dx=dx_next + dx_e + rb["dx"], dW_r=rb["dW_r"], dsigma=rb["dsigma"], dg=dg,
                 dx_expert=dx_e, dx_router=rb["dx"])
 

@@ -13,13 +13,13 @@ from oracle import unipool_oracle as O
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "hand_examples.json")
 
 
-def tiny_problem(seed=0, L=3, M=6, d=8, f=5, k=2, T=12, private=0, std=0.5, bias=False):
+def tiny_problem(seed=0, L=3, M=6, d=8, f=5, k=2, T=12, private=0, std=0.5, bias=False, mode="norm"):
     rng = np.random.default_rng(seed)
     m = private if private else M
     pool = dict(W_gate=rng.normal(0, std, (M, f, d)), W_up=rng.normal(0, std, (M, f, d)),
                 W_down=rng.normal(0, std, (M, d, f)))
     routers = [dict(W_r=rng.normal(0, std, (m, d)), sigma=1.0 + 0.1 * l,
-                    bias=(rng.normal(0, 0.3, m) if bias else None)) for l in range(L)]
+                    bias=(rng.normal(0, 0.3, m) if bias else None), mode=mode) for l in range(L)]
     x0 = rng.normal(0, 1, (T, d))
     up = rng.normal(0, 1, (T, d))
     views = [private * l for l in range(L)] if private else None
@@ -236,6 +236,60 @@ def test_aux_loss_identities():
     np.testing.assert_allclose(fb_now, fbar)
 
 
+# ---------------------------------------------------------------- softmax router (the paper's baseline router)
+def test_softmax_router_against_library_and_closed_forms():
+    from scipy.special import logsumexp, softmax
+    rng = np.random.default_rng(5)
+    z = rng.normal(0, 3, (40, 11))
+    z[3] += 700.0                                      # would overflow exp() without the max subtraction
+    s, lse = O.softmax_router_scores(z)
+    np.testing.assert_allclose(s, softmax(z, axis=1), rtol=1e-13, atol=0)
+    np.testing.assert_allclose(lse, logsumexp(z, axis=1), rtol=1e-13)
+    np.testing.assert_allclose(s.sum(1), 1.0, rtol=1e-13)
+    np.testing.assert_allclose(O.softmax_router_scores(z - 17.5)[0], s, rtol=1e-12)       # shift invariance
+    np.testing.assert_allclose(O.softmax_router_scores(np.full((2, 8), 0.3))[0], 1.0 / 8)  # equal logits
+    # two experts: the logistic function of the logit difference
+    z2 = rng.normal(0, 2, (9, 2))
+    np.testing.assert_allclose(O.softmax_router_scores(z2)[0][:, 0], 1 / (1 + np.exp(z2[:, 1] - z2[:, 0])), rtol=1e-13)
+    # exp is increasing: the softmax top-k is the top-k of the logits, gates are the probabilities
+    x = rng.normal(0, 1, (30, 6))
+    W = rng.normal(0, 1, (11, 6))
+    b = rng.normal(0, 1, 11)
+    r = O.route(x, W, 123.0, 456.0, 0.5, 3, bias=b, mode="softmax")   # sigma, c, eps play no part
+    zz = x @ W.T + b
+    np.testing.assert_array_equal(r["idx"], np.argsort(-zz, axis=1, kind="stable")[:, :3])
+    np.testing.assert_allclose(r["g"], np.take_along_axis(softmax(zz, axis=1), r["idx"].astype(np.int64), 1), rtol=1e-13)
+    np.testing.assert_allclose(r["S"].sum(), 30.0, rtol=1e-13)          # every token's probabilities sum to one
+    assert r["counts"].sum() == 30 * 3
+    # with probabilities, uniform routing reaches the Switch minimum of the balance loss: alpha
+    counts = np.full((2, 8), 5)
+    S = np.full((2, 8), 20 / 8.0)
+    loss, _, _ = O.pool_aux_loss(counts, S, 20, 2, 0.01)
+    assert loss == pytest.approx(0.01, rel=1e-13)
+
+
+def test_softmax_backward_is_the_textbook_jacobian():
+    rng = np.random.default_rng(6)
+    T, M, d, k = 5, 7, 4, 2
+    x = rng.normal(0, 1, (T, d))
+    W = rng.normal(0, 1, (M, d))
+    r = O.route(x, W, 1.0, 1.0, 1e-6, k, mode="softmax")
+    dg = rng.normal(0, 1, (T, k))
+    coef = rng.normal(0, 1, M)
+    rb = O.route_backward(x, W, 1.0, 1.0, 1e-6, r["z"], r["n"], r["idx"], dg, coef, mode="softmax")
+    for t in range(T):
+        ds = coef.copy()
+        for j in range(k):
+            ds[r["idx"][t, j]] += dg[t, j]
+        s = r["s"][t]
+        jac = np.diag(s) - np.outer(s, s)               # d s_i / d z_m
+        np.testing.assert_allclose(rb["dz"][t], jac.T @ ds, rtol=1e-12, atol=1e-15)
+    np.testing.assert_allclose(rb["dW_r"], sum(np.outer(rb["dz"][t], x[t]) for t in range(T)), rtol=1e-12)
+    np.testing.assert_allclose(rb["dx"], np.stack([W.T @ rb["dz"][t] for t in range(T)]), rtol=1e-12)
+    assert rb["dsigma"] == 0.0
+    np.testing.assert_allclose(rb["dz"].sum(1), 0.0, atol=1e-14)          # probabilities sum to a constant
+
+
 # ---------------------------------------------------------------- backward
 def _objective(x0, routers, pool, k, c, eps, alpha, up, views, forced, fbar_prev, n_view):
     caches = O.stack_forward(x0, routers, pool, k, c, eps, views, forced)
@@ -249,10 +303,11 @@ def _objective(x0, routers, pool, k, c, eps, alpha, up, views, forced, fbar_prev
     return float(np.sum(up * caches[-1]["x_next"]) + aux), [cc["idx"] for cc in caches]
 
 
-@pytest.mark.parametrize("private,bias", [(0, False), (0, True), (2, False)])
-def test_backward_matches_central_finite_differences(private, bias):
+@pytest.mark.parametrize("private,bias,mode", [(0, False, "norm"), (0, True, "norm"), (2, False, "norm"),
+                                               (0, True, "softmax"), (2, False, "softmax")])
+def test_backward_matches_central_finite_differences(private, bias, mode):
     pool, routers, x0, up, views = tiny_problem(seed=11, L=3, M=6, d=8, f=5, k=2, T=10,
-                                                private=private, bias=bias)
+                                                private=private, bias=bias, mode=mode)
     k, c, eps, alpha = 2, 1.9, 1e-6, 0.5          # a large alpha makes the balance term visible
     res = O.stack_objective_and_grads(x0, routers, pool, k, c, eps, alpha, up, views, n_view=private)
     base_idx = [cc["idx"] for cc in res["caches"]]
