@@ -149,7 +149,7 @@ def run_ours(args):
     small.close()
     del small
     st = UniPoolStack(L, d, f, M, k, T, cfg["dtype"], cfg["private"], c=c_val, eps=synth.EPS, alpha=synth.ALPHA,
-                      device=dev, deferred_wgrad=args.deferred_wgrad)
+                      device=dev, deferred_wgrad=args.deferred_wgrad, router=cfg.get("router", "norm"))
     st.load(inputs["pool"], inputs["routers"])
     tdt = st.tdtype
     x0_host = torch.from_numpy(inputs["x0"]).to(tdt).pin_memory()
@@ -331,7 +331,7 @@ def cpu_baseline(cfg, budget_tokens=2048, repeats=1):
         threads = len(os.sched_getaffinity(0))
     Ts = min(budget_tokens, cfg["T"])
     inputs = synth.make_inputs(cfg, seed=0, T=Ts, L=1)
-    pool, router = inputs["pool"], inputs["routers"][0]
+    pool, router = inputs["pool"], dict(inputs["routers"][0], mode=cfg.get("router", "norm"))
     k = cfg["k"]
     best = None
     for _ in range(repeats):

@@ -52,6 +52,12 @@ extern "C" {
 #define UNIPOOL_FP32 0
 #define UNIPOOL_BF16 1
 
+/* router_mode of a context */
+#define UNIPOOL_ROUTER_NORM    0      /* NormRouter, Eq. 7                          */
+#define UNIPOOL_ROUTER_SOFTMAX 1      /* softmax over the router's experts: the     */
+                                      /* conventional router of the baselines in    */
+                                      /* Sec. 5.1 and of the ablation of Sec. 5.3   */
+
 #define UNIPOOL_ROW_ALIGN 128         /* group starts in the permuted row space    */
 #define UNIPOOL_MAX_EXPERTS 512
 #define UNIPOOL_MAX_TOPK 8
@@ -79,6 +85,7 @@ typedef struct {
   int32_t dtype;        /* UNIPOOL_FP32 or UNIPOOL_BF16                          */
   float   eps;          /* epsilon of Eq. 7                                      */
   float   c;            /* calibration constant c of Eq. 7 (Alg. 1)              */
+  int32_t router_mode;  /* UNIPOOL_ROUTER_NORM or UNIPOOL_ROUTER_SOFTMAX         */
 } unipool_config;
 
 /* Rows a permuted buffer must have: max_tokens*top_k + pool_size*(ROW_ALIGN-1),
@@ -113,7 +120,11 @@ int unipool_check_status(unipool_ctx* ctx, unipool_stream stream);
  * out: idx [T,k] int32; gate [T,k] float; counts [n_experts] int32 (assignments
  *      per expert); score_sum [n_experts] float (sum over tokens of s, the
  *      numerator of P_i in Eq. 3); znorm [T] float; z_saved [T,n_experts] float
- *      (logits, kept for unipool_route_bwd).  All outputs are overwritten. */
+ *      (logits, kept for unipool_route_bwd).  All outputs are overwritten.
+ * A context of router_mode UNIPOOL_ROUTER_SOFTMAX scores with
+ *   s = exp(z - max z) / sum_j exp(z_j - max z)
+ * instead (sigma, c and eps play no part) and stores log sum_j exp(z_j) in
+ * znorm; selection, gates and statistics are taken from s in the same way. */
 int unipool_route(unipool_ctx* ctx, const void* x, int32_t T, const float* W_r, float sigma,
                   const float* bias, int32_t n_experts, int32_t* idx, float* gate,
                   int32_t* counts, float* score_sum, float* znorm, float* z_saved,
@@ -234,7 +245,9 @@ int unipool_pool_aux_loss(unipool_ctx* ctx, const int32_t* counts, const float* 
  *   dsigma += c sum ds u/(n+eps);  dW_r += dz^T x;  dx += dz W_r.
  * in : x [T,d]; W_r; sigma; znorm, z_saved, idx from unipool_route; dgate [T,k];
  *      dscore_coef [n_experts] or NULL.
- * out: dx [T,d] (ctx dtype) +=; dW_r [n_experts,d] float +=; dsigma (device float) +=. */
+ * out: dx [T,d] (ctx dtype) +=; dW_r [n_experts,d] float +=; dsigma (device float) +=.
+ * With router_mode UNIPOOL_ROUTER_SOFTMAX: s = exp(z - znorm) (znorm holds the
+ * log-sum-exp), q_t = sum_i ds s, dz[t,m] = s_m (ds_m - q_t); dsigma is left as it is. */
 int unipool_route_bwd(unipool_ctx* ctx, const void* x, int32_t T, const float* W_r, float sigma,
                       int32_t n_experts, const float* znorm, const float* z_saved,
                       const int32_t* idx, const float* dgate, const float* dscore_coef,

@@ -14,6 +14,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libunipool.so")
 
 FP32, BF16 = 0, 1
+ROUTER_NORM, ROUTER_SOFTMAX = 0, 1
 ROW_ALIGN = 128
 BWD_SKIP_WGRAD = 1
 WGRAD_OVERWRITE = 2
@@ -39,6 +40,7 @@ class Config(ctypes.Structure):
         ("d_model", ctypes.c_int32), ("d_ff", ctypes.c_int32), ("pool_size", ctypes.c_int32),
         ("top_k", ctypes.c_int32), ("n_layers", ctypes.c_int32), ("max_tokens", ctypes.c_int32),
         ("dtype", ctypes.c_int32), ("eps", ctypes.c_float), ("c", ctypes.c_float),
+        ("router_mode", ctypes.c_int32),
     ]
 
 
@@ -121,8 +123,8 @@ def _stream():
     return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
 
 
-def make_config(d_model, d_ff, pool_size, top_k, n_layers, max_tokens, dtype, eps, c):
-    return Config(d_model, d_ff, pool_size, top_k, n_layers, max_tokens, dtype, eps, c)
+def make_config(d_model, d_ff, pool_size, top_k, n_layers, max_tokens, dtype, eps, c, router_mode=0):
+    return Config(d_model, d_ff, pool_size, top_k, n_layers, max_tokens, dtype, eps, c, router_mode)
 
 
 def row_capacity(cfg):

@@ -87,6 +87,8 @@ static int validate_config(const unipool_config* c) {
   UP_REQUIRE(c->max_tokens >= 1 && (int64_t)c->max_tokens * c->top_k < (1ll << 30),
              UNIPOOL_ERR_UNSUPPORTED, "max_tokens*top_k must be in [1, 2^30)");
   UP_REQUIRE(c->eps >= 0.f && c->c > 0.f, UNIPOOL_ERR_INVALID_ARG, "eps must be >= 0 and c > 0");
+  UP_REQUIRE(c->router_mode == UNIPOOL_ROUTER_NORM || c->router_mode == UNIPOOL_ROUTER_SOFTMAX,
+             UNIPOOL_ERR_INVALID_ARG, "router_mode must be UNIPOOL_ROUTER_NORM or UNIPOOL_ROUTER_SOFTMAX");
   return UNIPOOL_OK;
 }
 

@@ -1,4 +1,4 @@
-// NormRouter forward (Eq. 7 + top-k, Sec. 4.3) and backward.
+// Router forward (NormRouter, Eq. 7, or softmax; top-k, Sec. 4.3) and backward.
 #include <cfloat>
 
 #include "common.cuh"
@@ -34,6 +34,7 @@ router_logits_kernel(const TX* __restrict__ x, const float* __restrict__ W_r,
 constexpr int kRouteWarps = 8;
 constexpr int kRouteTokensPerWarp = 4;
 
+template <bool SOFTMAX>
 __global__ void __launch_bounds__(kRouteWarps * 32)
 router_select_kernel(const float* __restrict__ z, int T, int M, int k, float sigma_c, float eps,
                      int32_t* __restrict__ idx, float* __restrict__ gate, float* __restrict__ znorm,
@@ -55,22 +56,48 @@ router_select_kernel(const float* __restrict__ z, int T, int M, int k, float sig
     const int t = t_begin + tt;
     if (t >= T) break;
     const float* zr = z + (int64_t)t * M;
-    float ss = 0.f;
-    for (int i = lane; i < M; i += 32) {
-      float v = zr[i];
-      my[i] = v;
-      ss = fmaf(v, v, ss);
-    }
+    if (SOFTMAX) {
+      // s = exp(z - max) / sum exp(z - max); the log-sum-exp goes where the NormRouter keeps ||z||
+      float mx = -INFINITY;
+      for (int i = lane; i < M; i += 32) {
+        float v = zr[i];
+        my[i] = v;
+        mx = fmaxf(mx, v);
+      }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-    const float n = sqrtf(ss);
-    const float den = n + eps;
-    for (int i = lane; i < M; i += 32) {
-      float s = sigma_c * fmaxf(0.f, my[i] / den);
-      my[i] = s;
-      wsum[warp * M + i] += s;
+      for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+      float tot = 0.f;
+      for (int i = lane; i < M; i += 32) {
+        float e = expf(my[i] - mx);
+        my[i] = e;
+        tot += e;
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, o);
+      for (int i = lane; i < M; i += 32) {
+        float s = my[i] / tot;
+        my[i] = s;
+        wsum[warp * M + i] += s;
+      }
+      if (lane == 0) znorm[t] = mx + logf(tot);
+    } else {
+      float ss = 0.f;
+      for (int i = lane; i < M; i += 32) {
+        float v = zr[i];
+        my[i] = v;
+        ss = fmaf(v, v, ss);
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+      const float n = sqrtf(ss);
+      const float den = n + eps;
+      for (int i = lane; i < M; i += 32) {
+        float s = sigma_c * fmaxf(0.f, my[i] / den);
+        my[i] = s;
+        wsum[warp * M + i] += s;
+      }
+      if (lane == 0) znorm[t] = n;
     }
-    if (lane == 0) znorm[t] = n;
     __syncwarp();
     for (int j = 0; j < k; ++j) {
       float bv = -INFINITY;
@@ -152,9 +179,10 @@ int route_launch(unipool_ctx* ctx, const void* x, int T, const float* W_r, float
   const int per_block = kRouteWarps * kRouteTokensPerWarp;
   const int blocks = (T + per_block - 1) / per_block;
   const size_t smem = (size_t)(2 * kRouteWarps * M) * sizeof(float) + (size_t)M * sizeof(int);
+  auto kern = ctx->cfg.router_mode == UNIPOOL_ROUTER_SOFTMAX ? router_select_kernel<true> : router_select_kernel<false>;
   if (smem > 48 * 1024)
-    UP_CUDA(cudaFuncSetAttribute(router_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  router_select_kernel<<<blocks, kRouteWarps * 32, smem, s>>>(
+    UP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  kern<<<blocks, kRouteWarps * 32, smem, s>>>(
       z_saved, T, M, k, sigma * ctx->cfg.c, ctx->cfg.eps, idx, gate, znorm, counts, score_sum,
       ctx->ws.route_counts, ctx->ws.route_sums, ctx->ws.tickets + 0);
   UP_LAUNCH_CHECK();
@@ -163,6 +191,7 @@ int route_launch(unipool_ctx* ctx, const void* x, int T, const float* W_r, float
 
 // ---------------------------------------------------------------- backward
 // dz from (z, n, idx, dgate, coef); one warp per token.
+template <bool SOFTMAX>
 __global__ void __launch_bounds__(256)
 router_dz_kernel(const float* __restrict__ z, const float* __restrict__ znorm,
                  const int32_t* __restrict__ idx, const float* __restrict__ dgate,
@@ -189,7 +218,7 @@ router_dz_kernel(const float* __restrict__ z, const float* __restrict__ znorm,
         float dj = __shfl_sync(0xffffffffu, my_dg, j);
         if (ej == i) ds += dj;
       }
-      if (i < M) q = fmaf(ds, fmaxf(zr[i], 0.f), q);
+      if (i < M) q = fmaf(ds, SOFTMAX ? expf(zr[i] - n) : fmaxf(zr[i], 0.f), q);
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
@@ -206,10 +235,11 @@ router_dz_kernel(const float* __restrict__ z, const float* __restrict__ znorm,
       if (i < M) {
         float zi = zr[i];
         float v = n > 0.f ? scale * ((zi > 0.f ? ds / ne : 0.f) - zi * qn) : 0.f;
+        if (SOFTMAX) v = expf(zi - n) * (ds - q);          // n holds log sum exp(z)
         dz[(int64_t)t * M + i] = v;
       }
     }
-    dsig_part = c * q / ne;
+    dsig_part = SOFTMAX ? 0.f : c * q / ne;
   }
   __shared__ float part[8];
   if (lane == 0) part[warp] = dsig_part;
@@ -288,9 +318,9 @@ int route_bwd_launch(unipool_ctx* ctx, const void* x, int T, const float* W_r, f
   float* dz = ctx->ws.dz;
   {
   PhaseTimer pt(ctx, UNIPOOL_PH_ROUTE_BWD_DZ, 1, s);
-  router_dz_kernel<<<(T + 7) / 8, 256, 0, s>>>(z_saved, znorm, idx, dgate, coef, T, M, k, sigma,
-                                               ctx->cfg.c, ctx->cfg.eps, dz, dsigma,
-                                               ctx->ws.dsigma_acc, ctx->ws.tickets + 1);
+  auto kern = ctx->cfg.router_mode == UNIPOOL_ROUTER_SOFTMAX ? router_dz_kernel<true> : router_dz_kernel<false>;
+  kern<<<(T + 7) / 8, 256, 0, s>>>(z_saved, znorm, idx, dgate, coef, T, M, k, sigma, ctx->cfg.c,
+                                   ctx->cfg.eps, dz, dsigma, ctx->ws.dsigma_acc, ctx->ws.tickets + 1);
   UP_LAUNCH_CHECK();
   }
   dim3 g2((T + kSimtTile - 1) / kSimtTile, d / kSimtTile);

@@ -70,7 +70,7 @@ __device__ __forceinline__ void route_timeout(const RouteParams& p, volatile int
   }
 }
 
-template <int KMAX>
+template <int KMAX, bool SOFTMAX>
 __global__ void __launch_bounds__(kThreads, 1)
 route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW,
                 const __grid_constant__ CUtensorMap tmZ, const RouteParams p) {
@@ -177,10 +177,11 @@ route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     tc::tc_fence_after_sync();
     const uint32_t t_row = tmem_base + (static_cast<uint32_t>(warp * 32) << 16);
     if (ok) {
-      // pass 1: logits (+ bias) -> z_saved, squared norm.  With a 16-byte row pitch (M % 4 == 0) the
+      // pass 1: logits (+ bias) -> z_saved, squared norm (softmax: running maximum and the sum of
+      // exponentials relative to it).  With a 16-byte row pitch (M % 4 == 0) the
       // 32 x 32 chunk is staged in shared memory (128-byte swizzle, conflict-free) and leaves by a
       // TMA store, which clips it at M columns and T rows.
-      float ss = 0.f;
+      float ss = 0.f, mx = -INFINITY;
       float* zrow = p.z_saved + (int64_t)t * M;
       const bool vec = (M & 3) == 0;
       uint8_t* my_stage = zstage + warp * 2 * 4096;
@@ -192,8 +193,19 @@ route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         float z[32];
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
-          z[i] = c0 + i < M ? __uint_as_float(rr[i]) + sbias[c0 + i] : 0.f;
-          ss = fmaf(z[i], z[i], ss);
+          z[i] = c0 + i < M ? __uint_as_float(rr[i]) + sbias[c0 + i] : (SOFTMAX ? -INFINITY : 0.f);
+          if (!SOFTMAX) ss = fmaf(z[i], z[i], ss);
+        }
+        if (SOFTMAX) {
+          float cm = z[0];
+#pragma unroll
+          for (int i = 1; i < 32; ++i) cm = fmaxf(cm, z[i]);
+          cm = fmaxf(cm, mx);
+          float part = 0.f;
+#pragma unroll
+          for (int i = 0; i < 32; ++i) part += expf(z[i] - cm);
+          ss = ss * expf(mx - cm) + part;                 // the first chunk rescales an empty sum
+          mx = cm;
         }
         if (vec) {
           uint8_t* buf = my_stage + (nstore++ & 1) * 4096;
@@ -215,8 +227,9 @@ route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
             if (c0 + i < M) zrow[c0 + i] = z[i];
         }
       }
-      const float n = sqrtf(ss);
-      const float scale = ss > 0.f ? p.sigma_c / (n + p.eps) : 0.f;   // a zero logit vector scores zero
+      const float n = SOFTMAX ? mx + logf(ss) : sqrtf(ss);           // softmax keeps log sum exp(z) here
+      // NormRouter: a zero logit vector scores zero.  Softmax: 1 / sum of exponentials.
+      const float scale = SOFTMAX ? 1.f / ss : (ss > 0.f ? p.sigma_c / (n + p.eps) : 0.f);
       if (live) p.znorm[t] = n;
       // pass 2: scores, top-k (score descending, expert index ascending), per-expert score sums
       float tv[KMAX];
@@ -232,7 +245,7 @@ route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         for (int i = 0; i < 32; ++i) {
           const int e = c0 + i;
           const float z = __uint_as_float(rr[i]) + sbias[e < M ? e : 0];
-          const float s = e < M ? scale * fmaxf(z, 0.f) : 0.f;
+          const float s = e < M ? scale * (SOFTMAX ? expf(z - mx) : fmaxf(z, 0.f)) : 0.f;
           float key = s == s ? s : -FLT_MAX;              // NaN scores sort last but stay selectable
           if (e >= M) key = -INFINITY;                    // never selected
           // Insert behind every entry that is >= key (equal keys keep the lower index in front) and
@@ -329,7 +342,8 @@ route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   }
 }
 
-// dz of the NormRouter derivative as bf16 [T, Mp] (columns >= M are zero); four lanes per token.
+// dz of the router's derivative as bf16 [T, Mp] (columns >= M are zero); four lanes per token.
+template <bool SOFTMAX>
 __global__ void __launch_bounds__(256)
 router_dz16_kernel(const float* __restrict__ z, const float* __restrict__ znorm, const int32_t* __restrict__ idx,
                    const float* __restrict__ dgate, const float* __restrict__ coef, int T, int M, int Mp, int k,
@@ -354,11 +368,11 @@ router_dz16_kernel(const float* __restrict__ z, const float* __restrict__ znorm,
       if (e_sel[j] == i) ds += dg_sel[j];
     return ds;
   };
+  const float n = znorm[t];                       // ||z||; softmax: log sum exp(z)
   float q = 0.f;
-  for (int i = sub; i < M; i += 4) q = fmaf(ds_of(i), fmaxf(zr[i], 0.f), q);
+  for (int i = sub; i < M; i += 4) q = fmaf(ds_of(i), SOFTMAX ? expf(zr[i] - n) : fmaxf(zr[i], 0.f), q);
   q += __shfl_xor_sync(0xffffffffu, q, 1);
   q += __shfl_xor_sync(0xffffffffu, q, 2);
-  const float n = znorm[t];
   const float ne = n + eps;
   const float scale = sigma * c;
   const float qn = n > 0.f ? q / (n * ne * ne) : 0.f;
@@ -366,14 +380,16 @@ router_dz16_kernel(const float* __restrict__ z, const float* __restrict__ znorm,
     __nv_bfloat16* out = dz16 + (int64_t)t * Mp;
     for (int i = sub; i < Mp; i += 4) {
       float v = 0.f;
-      if (i < M && n > 0.f) {
+      if (SOFTMAX) {
+        if (i < M) v = expf(zr[i] - n) * (ds_of(i) - q);
+      } else if (i < M && n > 0.f) {
         const float zi = zr[i];
         v = scale * ((zi > 0.f ? ds_of(i) / ne : 0.f) - zi * qn);
       }
       out[i] = __float2bfloat16_rn(v);
     }
   }
-  float part = (live && sub == 0) ? c * q / ne : 0.f;
+  float part = (live && sub == 0 && !SOFTMAX) ? c * q / ne : 0.f;
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
   __shared__ float wpart[8];
@@ -443,13 +459,11 @@ int route_tc_launch(unipool_ctx* ctx, const void* x, int T, const float* W_r, fl
   PhaseTimer pt(ctx, UNIPOOL_PH_ROUTE_SELECT, 1, s);
   const size_t smem = (size_t)p.stages * stage_bytes + tail_bytes + 1024;
   const int grid = (T + kTile - 1) / kTile;
-  if (k <= 2) {
-    UP_CUDA(cudaFuncSetAttribute(route_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    route_tc_kernel<2><<<grid, kThreads, smem, s>>>(tmX, tmW, tmZ, p);
-  } else {
-    UP_CUDA(cudaFuncSetAttribute(route_tc_kernel<UNIPOOL_MAX_TOPK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    route_tc_kernel<UNIPOOL_MAX_TOPK><<<grid, kThreads, smem, s>>>(tmX, tmW, tmZ, p);
-  }
+  const bool softmax = ctx->cfg.router_mode == UNIPOOL_ROUTER_SOFTMAX;
+  auto kern = k <= 2 ? (softmax ? route_tc_kernel<2, true> : route_tc_kernel<2, false>)
+                     : (softmax ? route_tc_kernel<UNIPOOL_MAX_TOPK, true> : route_tc_kernel<UNIPOOL_MAX_TOPK, false>);
+  UP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  kern<<<grid, kThreads, smem, s>>>(tmX, tmW, tmZ, p);
   UP_LAUNCH_CHECK();
   return UNIPOOL_OK;
 }
@@ -465,7 +479,8 @@ int route_bwd_tc_launch(unipool_ctx* ctx, const void* x, int T, const float* W_r
     PhaseTimer pt(ctx, UNIPOOL_PH_ROUTE_BWD_DZ, 2, s);
     if ((rc = router_split_launch(ctx, W_r, M, s)) != UNIPOOL_OK) return rc;   // term 0 = bf16(W_r)
     const int64_t threads = (int64_t)T * 4;
-    router_dz16_kernel<<<(int)((threads + 255) / 256), 256, 0, s>>>(
+    auto kern = ctx->cfg.router_mode == UNIPOOL_ROUTER_SOFTMAX ? router_dz16_kernel<true> : router_dz16_kernel<false>;
+    kern<<<(int)((threads + 255) / 256), 256, 0, s>>>(
         z_saved, znorm, idx, dgate, coef, T, M, Mp, k, sigma, ctx->cfg.c, ctx->cfg.eps, dz16, dsigma,
         ctx->ws.dsigma_acc, ctx->ws.tickets + 1);
     UP_LAUNCH_CHECK();

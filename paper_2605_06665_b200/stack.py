@@ -13,7 +13,9 @@ owns pool experts [E*l, E*(l+1)) (the layer-private layout of Eq. 1); with
 consecutive groups of L/G layers, group g sharing pool experts [g*M/G, (g+1)*M/G)
 with its own balance loss (Eq. 5 over the group's layers; G = 1 is UniPool, G = L
 the private layout).  In the private layout the
-balance loss is the per-layer loss of Eq. 3 summed over layers.
+balance loss is the per-layer loss of Eq. 3 summed over layers.  ``router="softmax"``
+replaces the NormRouter of Eq. 7 by the conventional softmax router of the paper's
+baselines (Sec. 5.1) in every layer.
 """
 from __future__ import annotations
 
@@ -25,7 +27,7 @@ from . import binding as B
 
 class UniPoolStack:
     def __init__(self, L, d, f, M, k, T, dtype="bf16", private=0, c=1.0, eps=1e-6, alpha=1e-2,
-                 device="cuda", deferred_wgrad=False, recompute=False, groups=None):
+                 device="cuda", deferred_wgrad=False, recompute=False, groups=None, router="norm"):
         self.L, self.d, self.f, self.M, self.k, self.T = L, d, f, M, k, T
         if groups is None:
             groups = L if private else 1
@@ -43,7 +45,11 @@ class UniPoolStack:
         self.deferred_wgrad = deferred_wgrad and self.Lg > 1 and not recompute
         self.device = torch.device(device)
         self.tdtype = torch.bfloat16 if dtype == "bf16" else torch.float32
-        self.cfg = B.make_config(d, f, M, k, L, T, B.BF16 if dtype == "bf16" else B.FP32, eps, c)
+        if router not in ("norm", "softmax"):
+            raise ValueError("router must be 'norm' or 'softmax'")
+        self.router = router
+        self.cfg = B.make_config(d, f, M, k, L, T, B.BF16 if dtype == "bf16" else B.FP32, eps, c,
+                                 B.ROUTER_SOFTMAX if router == "softmax" else B.ROUTER_NORM)
         self.ctx = B.Context(self.cfg, self.device)
         cap = self.ctx.row_capacity
         self.cap = cap

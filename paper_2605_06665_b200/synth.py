@@ -29,6 +29,9 @@ CONFIGS = {
     "tiny_fp32":      dict(L=4,  d=256,  f=512,  M=16,  k=2, T=512,   dtype="fp32", private=0, zipf_beta=0.0),
     "182m":           dict(L=12, d=768,  f=2048, M=96,  k=2, T=16384, dtype="bf16", private=0, zipf_beta=0.0),
     "182m_vanilla":   dict(L=12, d=768,  f=2048, M=96,  k=2, T=16384, dtype="bf16", private=8, zipf_beta=0.0),
+    # the paper's own baseline (Sec. 5.1): 8 private experts per layer, top-1, softmax router
+    "182m_vanilla_softmax": dict(L=12, d=768, f=2048, M=96, k=1, T=16384, dtype="bf16", private=8, zipf_beta=0.0,
+                                 router="softmax"),
     "182m_pool40":    dict(L=12, d=768,  f=2048, M=40,  k=2, T=16384, dtype="bf16", private=0, zipf_beta=0.0),
     "978m":           dict(L=24, d=1536, f=4096, M=192, k=2, T=32768, dtype="bf16", private=0, zipf_beta=0.0),
     "978m_pool128":   dict(L=24, d=1536, f=4096, M=128, k=2, T=32768, dtype="bf16", private=0, zipf_beta=0.0),

@@ -37,33 +37,40 @@ def rel_max(got, ref):
     return num / den if den > 0 else num
 
 
-def margin_safe(z, k, tol=MARGIN):
+def _keys(z, mode):
+    """What the top-k orders by, up to an increasing map: max(z, 0) for the NormRouter, z for softmax."""
+    return f64(z) if mode == "softmax" else np.maximum(f64(z), 0.0)
+
+
+def margin_safe(z, k, tol=MARGIN, mode="norm"):
     """Per token: is the top-k SET forced (k-th and (k+1)-th largest of max(z,0) differ
     by more than tol, or both are exactly zero scores with no logit within tol of 0),
     and is the slot ORDER forced (adjacent selected scores differ by more than tol)."""
-    u = np.maximum(f64(z), 0.0)
+    u = _keys(z, mode)
     srt = -np.sort(-u, axis=1)
     M = z.shape[1]
     if k < M:
         gap = srt[:, k - 1] - srt[:, k]
-        near_zero = (np.abs(f64(z)) < tol).any(axis=1)
+        near_zero = (np.abs(f64(z)) < tol).any(axis=1) & (mode != "softmax")
         set_safe = (gap > tol) | ((srt[:, k - 1] == 0) & ~near_zero)
         # zero-score picks are decided by index; they are safe only if no logit can flip sign
         set_safe &= ~((srt[:, k - 1] == 0) & near_zero)
+        if mode == "softmax":                          # every key is a logit: only the gap decides
+            set_safe = gap > tol
     else:
         set_safe = np.ones(z.shape[0], bool)
     if k > 1:
         adj = srt[:, :k - 1] - srt[:, 1:k]
-        both_zero = (srt[:, :k - 1] == 0) & (srt[:, 1:k] == 0)
+        both_zero = (srt[:, :k - 1] == 0) & (srt[:, 1:k] == 0) & (mode != "softmax")
         order_safe = ((adj > tol) | both_zero).all(axis=1)
     else:
         order_safe = np.ones(z.shape[0], bool)
     return set_safe, order_safe & set_safe
 
 
-def check_routing(idx_gpu, z_ref, idx_ref, k):
+def check_routing(idx_gpu, z_ref, idx_ref, k, mode="norm"):
     """Bit-exact where the margin forces the decision; a valid top-k elsewhere."""
-    set_safe, order_safe = margin_safe(z_ref, k)
+    set_safe, order_safe = margin_safe(z_ref, k, mode=mode)
     assert (idx_gpu[order_safe] == idx_ref[order_safe]).all(), "routing differs on margin-safe tokens"
     only_set = set_safe & ~order_safe
     assert (np.sort(idx_gpu[only_set], axis=1) == np.sort(idx_ref[only_set], axis=1)).all()
@@ -72,7 +79,7 @@ def check_routing(idx_gpu, z_ref, idx_ref, k):
     assert ((idx_gpu >= 0) & (idx_gpu < M)).all()
     srt = np.sort(idx_gpu, axis=1)
     assert (srt[:, 1:] != srt[:, :-1]).all() if k > 1 else True
-    u = np.maximum(f64(z_ref), 0.0)
+    u = _keys(z_ref, mode)
     kth = -np.sort(-u, axis=1)[:, k - 1]
     picked = np.take_along_axis(u, idx_gpu.astype(np.int64), axis=1)
     assert (picked >= kth[:, None] - MARGIN).all()
@@ -86,13 +93,14 @@ def build_stack(cfg, inputs, T=None, L=None, deferred_wgrad=False, c=None):
     m = synth.router_width(cfg)
     c = calib_c(m, cfg["k"]) if c is None else c
     st = UniPoolStack(L, cfg["d"], cfg["f"], cfg["M"], cfg["k"], T, cfg["dtype"], cfg["private"], c=c,
-                      eps=synth.EPS, alpha=synth.ALPHA, deferred_wgrad=deferred_wgrad, groups=cfg.get("groups"))
+                      eps=synth.EPS, alpha=synth.ALPHA, deferred_wgrad=deferred_wgrad, groups=cfg.get("groups"),
+                      router=cfg.get("router", "norm"))
     st.load(inputs["pool"], inputs["routers"][:L])
     return st
 
 
-def oracle_params(inputs, L):
+def oracle_params(inputs, L, mode="norm"):
     pool = {n: f64(w) for n, w in inputs["pool"].items()}
-    routers = [dict(W_r=f64(r["W_r"]), sigma=float(r["sigma"]),
+    routers = [dict(W_r=f64(r["W_r"]), sigma=float(r["sigma"]), mode=mode,
                     bias=None if r["bias"] is None else f64(r["bias"])) for r in inputs["routers"][:L]]
     return pool, routers

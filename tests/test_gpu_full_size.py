@@ -43,6 +43,7 @@ def sampled_experts(total_counts, rng):
 
 @pytest.mark.parametrize("name,L", [
     ("182m", None), ("182m_vanilla", None), ("182m_pool40", None), ("fine_zipf", None),
+    ("182m_vanilla_softmax", None),
     ("978m", 2),            # full layer shape and pool; two layers keep the host-side set-up affordable
 ])
 def test_full_size_sampled_parity(name, L):
@@ -51,6 +52,7 @@ def test_full_size_sampled_parity(name, L):
     L = cfg["L"] if L is None else L
     T, k, d, f, M = cfg["T"], cfg["k"], cfg["d"], cfg["f"], cfg["M"]
     m = synth.router_width(cfg)
+    mode = cfg.get("router", "norm")
     inputs = synth.make_inputs(cfg, seed=0, L=L)
     st = build_stack(cfg, inputs, L=L, deferred_wgrad=True)
     pool = inputs["pool"]                                   # float32 holding bf16 values; products run in float64
@@ -67,11 +69,12 @@ def test_full_size_sampled_parity(name, L):
         torch.cuda.synchronize()
         x_l = f64(to_np(st.x[l]))
         xs.append(x_l)
-        ref = O.route(x_l, routers[l]["W_r"], routers[l]["sigma"], c, eps, k, routers[l]["bias"])
+        ref = O.route(x_l, routers[l]["W_r"], routers[l]["sigma"], c, eps, k, routers[l]["bias"], mode=mode)
         idx_gpu = to_np(st.idx[l])
-        check_routing(idx_gpu, ref["z"], ref["idx"], k)
+        check_routing(idx_gpu, ref["z"], ref["idx"], k, mode)
         assert rel_max(to_np(st.z[l]), ref["z"]) < 1e-5
-        ref = O.route(x_l, routers[l]["W_r"], routers[l]["sigma"], c, eps, k, routers[l]["bias"], forced_idx=idx_gpu)
+        ref = O.route(x_l, routers[l]["W_r"], routers[l]["sigma"], c, eps, k, routers[l]["bias"], forced_idx=idx_gpu,
+                      mode=mode)
         assert rel_max(to_np(st.gate[l]), ref["g"]) < 1e-5
         assert (to_np(st.counts[l]) == ref["counts"]).all() and ref["counts"].sum() == T * k
         assert rel_max(to_np(st.score_sum[l]), ref["S"]) < 1e-5
@@ -131,7 +134,7 @@ def test_full_size_sampled_parity(name, L):
         dx_e, dg = O.expert_path_backward(xs[l], r["idx"], r["g"], pool, dxn, base, tokens=tokens)
         assert rel_max(to_np(st.dgate)[tokens], dg) < TOL
         rb = O.route_backward(xs[l][tokens], routers[l]["W_r"], routers[l]["sigma"], c, eps, r["z"][tokens],
-                              r["n"][tokens], r["idx"][tokens], dg, coefs[l])
+                              r["n"][tokens], r["idx"][tokens], dg, coefs[l], mode=mode)
         got = f64(to_np(dx_out[torch.from_numpy(tokens).cuda()]))
         assert rel_max(got, dxn[tokens] + dx_e + rb["dx"]) < TOL
         if l in experts:

@@ -32,7 +32,8 @@ def run_layer_checks(cfg, T, L, seed=0, zero_grad_check=True):
     st = build_stack(cfg, inputs, T=T, L=L)
     tol = TOL[cfg["dtype"]]
     k, m, M = cfg["k"], synth.router_width(cfg), cfg["M"]
-    pool, routers = oracle_params(inputs, L)
+    mode = cfg.get("router", "norm")
+    pool, routers = oracle_params(inputs, L, mode)
     c, eps, alpha = st.c, synth.EPS, synth.ALPHA
     st.x[0].copy_(torch.from_numpy(inputs["x0"]))
     caches = []
@@ -40,13 +41,14 @@ def run_layer_checks(cfg, T, L, seed=0, zero_grad_check=True):
         st.forward_layer(l)
         torch.cuda.synchronize()
         x_l = f64(to_np(st.x[l]))
-        ref = O.route(x_l, routers[l]["W_r"], routers[l]["sigma"], c, eps, k, routers[l]["bias"])
+        ref = O.route(x_l, routers[l]["W_r"], routers[l]["sigma"], c, eps, k, routers[l]["bias"], mode=mode)
         idx_gpu = to_np(st.idx[l])
-        set_safe, order_safe = check_routing(idx_gpu, ref["z"], ref["idx"], k)
+        set_safe, order_safe = check_routing(idx_gpu, ref["z"], ref["idx"], k, mode)
         assert rel_max(to_np(st.z[l]), ref["z"]) < 1e-5
         assert rel_max(to_np(st.znorm[l]), ref["n"]) < 1e-5
         # everything downstream is compared with the GPU's own (valid) routing decision
-        ref = O.route(x_l, routers[l]["W_r"], routers[l]["sigma"], c, eps, k, routers[l]["bias"], forced_idx=idx_gpu)
+        ref = O.route(x_l, routers[l]["W_r"], routers[l]["sigma"], c, eps, k, routers[l]["bias"], forced_idx=idx_gpu,
+                      mode=mode)
         assert rel_max(to_np(st.gate[l]), ref["g"]) < 1e-5
         assert (to_np(st.counts[l]) == ref["counts"]).all()
         assert to_np(st.counts[l]).sum() == T * k
@@ -115,7 +117,7 @@ def run_layer_checks(cfg, T, L, seed=0, zero_grad_check=True):
         dx_e, dg = O.expert_path_backward(cc["x"], cc["idx"], cc["g"], pool, dxn, base, pool_grad)
         assert rel_max(to_np(st.dgate), dg) < tol
         rb = O.route_backward(cc["x"], routers[l]["W_r"], routers[l]["sigma"], c, eps, cc["z"], cc["n"],
-                              cc["idx"], dg, coefs[l])
+                              cc["idx"], dg, coefs[l], mode=mode)
         assert rel_max(to_np(dx_out), dxn + dx_e + rb["dx"]) < tol
         assert rel_max(to_np(st.dW_r[l]), rb["dW_r"]) < tol
         # dsigma is a signed sum over all (token, expert) terms: the bound scales with the sum of
@@ -165,6 +167,23 @@ def test_small_fp32_shapes(kw, T):
 def test_small_bf16_shapes(kw, T):
     cfg = small_cfg(**kw)
     run_layer_checks(cfg, T, cfg["L"], seed=4)
+
+
+@pytest.mark.parametrize("kw,T", [
+    (dict(router="softmax"), 300),                                            # fp32, shared pool, top-2
+    (dict(router="softmax", M=24, k=1, private=8, L=3), 260),                 # the paper's baseline: private experts, top-1
+    (dict(router="softmax", M=33, k=3, zipf_beta=2.0), 150),                  # skewed logits, ragged width
+    (dict(router="softmax", dtype="bf16", d=256, f=256, M=96, k=2), 700),     # tensor-core router
+    (dict(router="softmax", dtype="bf16", d=128, f=128, M=10, k=1), 333),     # unaligned logit rows
+    (dict(router="softmax", dtype="bf16", d=128, f=128, M=384, k=8, zipf_beta=0.4), 400),
+    (dict(router="softmax", dtype="bf16", d=256, f=256, M=24, k=1, private=8, L=3), 520),
+])
+def test_softmax_router_mode(kw, T):
+    """The conventional softmax router (the baselines of Sec. 5.1, the ablation rows of Sec. 5.3)
+    through the same calls: probabilities as scores and gates, the same selection, statistics and
+    balance loss, and its own derivative."""
+    cfg = small_cfg(**kw)
+    run_layer_checks(cfg, T, cfg["L"], seed=6)
 
 
 def test_tiny_fp32_end_to_end():
