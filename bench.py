@@ -174,13 +174,19 @@ def run_ours(args):
         sync_all()
         return dp.max_over_ranks(e0.elapsed_time(e1), world, dev)
 
+    # --grad-exchange: the step is one data-parallel replica's (statistics and gradients summed over
+    # the ranks, the pool's dW_down travelling while dW_gu is computed); issued eagerly
+    exchange = dp.GradientExchange(world) if args.grad_exchange else None
+    if exchange is not None:
+        args.graph = False
+
     def device_step():
         # the step's first weight-gradient contribution overwrites the fp32 pool gradient, so it
         # needs no zeroing; the (small) router gradients are zeroed inside the step
-        st.step(x0, up, accumulate=False)
+        st.step(x0, up, accumulate=False, exchange=exchange)
 
     def e2e_step():
-        st.step(x0_host, up_host, accumulate=False)   # H2D copies of this step's inputs from pinned memory
+        st.step(x0_host, up_host, accumulate=False, exchange=exchange)   # H2D copies of this step's inputs from pinned memory
         xL_host.copy_(st.x[L], non_blocking=True)
         loss_host.copy_(st.loss, non_blocking=True)
 
@@ -294,6 +300,7 @@ def run_ours(args):
         "config": {"workload": args.workload, "layers": L, "d_model": d, "d_ff": f, "pool_experts": M, "top_k": k,
                    "tokens_per_gpu": T, "layout": "private" if cfg["private"] else "shared_pool",
                    "deferred_wgrad": bool(st.deferred_wgrad), "cuda_graph": bool(args.graph),
+                   "grad_exchange": bool(args.grad_exchange),
                    "l2": "working set per step (weights + saved activations, several GB) exceeds the 126 MB L2",
                    "norm_router_c": c_val},
         "clocks": clocks,
@@ -390,6 +397,9 @@ def main():
                          "backward instead of contracting all layers' rows per expert in one pass at the end")
     ap.add_argument("--cpu-tokens", type=int, default=16384, help="token sample of the CPU-oracle baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--grad-exchange", action="store_true",
+                    help="sum routing statistics and gradients over the ranks inside the step (data-parallel "
+                         "training step); off: the ranks run independent token shards")
     ap.add_argument("--no-graph", dest="graph", action="store_false",
                     help="issue every library call of a step eagerly instead of replaying one CUDA graph")
     ap.add_argument("--kernels-only", action="store_true",

@@ -219,7 +219,10 @@ int unipool_expert_bwd(unipool_ctx* ctx, const void* dy, int32_t T, const int32_
  * the per-layer accumulation of unipool_expert_bwd up to summation order).
  * The per-layer operands are slices of stacked buffers: layer l's Xp is
  * Xp + l*layer_stride_rows*d elements, likewise A, dYp, dGU; offsets is
- * [n_layers, n_experts+1].  flags: 0 (dW +=) or UNIPOOL_WGRAD_OVERWRITE (dW =). */
+ * [n_layers, n_experts+1].  flags: 0 (dW +=) or UNIPOOL_WGRAD_OVERWRITE (dW =).
+ * One of dW_gu, dW_down may be NULL: only the other product is then computed
+ * (its operands alone are read), e.g. to start exchanging dW_down between
+ * data-parallel replicas while dW_gu is still being computed. */
 int unipool_pool_wgrad(unipool_ctx* ctx, int32_t n_layers, int64_t layer_stride_rows,
                        const int32_t* offsets, const void* Xp, const void* A, const void* dYp,
                        const void* dGU, int32_t expert_base, int32_t n_experts, float* dW_gu,

@@ -375,7 +375,8 @@ def zeros_like_pool(pool):
 
 
 def stack_objective_and_grads(x0, routers, pool, k, c, eps, alpha, upstream, views=None,
-                              forced_idx=None, fbar_prev=None, n_view=None, aux_groups=None):
+                              forced_idx=None, fbar_prev=None, n_view=None, aux_groups=None,
+                              replica_stats=None):
     """J = sum(upstream * x_L) + balance loss, and dJ/d(everything).
 
     UniPool (views None): balance loss = Eq. 5 over all L layers.  Layer-private
@@ -384,6 +385,10 @@ def stack_objective_and_grads(x0, routers, pool, k, c, eps, alpha, upstream, vie
     layers of every group; each group is a pool of its own, so its balance loss is Eq. 5 over the
     group's layers and experts (G = L gives sum_l Eq. 3, G = 1 gives Eq. 5).
     Routing decisions and f-bar are constants of the derivative.
+    Data-parallel replicas (App. D trains data parallel; the batch of Eqs. 3-5 is then the union of
+    the replicas' tokens): ``replica_stats(counts, S) -> (counts, S, T)`` returns the statistics summed
+    over all replicas and the total token count; the balance loss returned is the whole batch's, the
+    gradients are this replica's share (their sum over replicas is the whole batch's gradient).
     Returns dict(J, loss_aux, caches, pool_grad, router_grads [L], dx0).
     """
     L = len(routers)
@@ -391,6 +396,8 @@ def stack_objective_and_grads(x0, routers, pool, k, c, eps, alpha, upstream, vie
     caches = stack_forward(x0, routers, pool, k, c, eps, views, forced_idx)
     counts = np.stack([cch["counts"] for cch in caches])
     S = np.stack([cch["S"] for cch in caches])
+    if replica_stats is not None:
+        counts, S, T = replica_stats(counts, S)
     if aux_groups is not None:
         loss_aux = 0.0
         coefs = [None] * L

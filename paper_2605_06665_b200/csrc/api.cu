@@ -284,8 +284,10 @@ int unipool_pool_wgrad(unipool_ctx* ctx, int32_t n_layers, int64_t layer_stride_
   UP_REQUIRE(n_layers >= 1, UNIPOOL_ERR_INVALID_ARG, "n_layers must be >= 1");
   UP_REQUIRE(layer_stride_rows >= 0 && layer_stride_rows % UNIPOOL_ROW_ALIGN == 0,
              UNIPOOL_ERR_INVALID_ARG, "layer_stride_rows must be a multiple of %d", UNIPOOL_ROW_ALIGN);
-  CHECK_PTR(offsets); CHECK_PTR(Xp); CHECK_PTR(A); CHECK_PTR(dYp); CHECK_PTR(dGU);
-  CHECK_PTR(dW_gu); CHECK_PTR(dW_down);
+  CHECK_PTR(offsets);
+  UP_REQUIRE(dW_gu != nullptr || dW_down != nullptr, UNIPOOL_ERR_INVALID_ARG, "dW_gu and dW_down are both NULL");
+  if (dW_gu != nullptr) { CHECK_PTR(Xp); CHECK_PTR(dGU); }
+  if (dW_down != nullptr) { CHECK_PTR(A); CHECK_PTR(dYp); }
   UP_REQUIRE((flags & ~UNIPOOL_WGRAD_OVERWRITE) == 0, UNIPOOL_ERR_INVALID_ARG, "unknown flags 0x%x", flags);
   PoolWgradArgs a{n_layers, layer_stride_rows, offsets, Xp, A, dYp, dGU, expert_base, n_experts,
                   dW_gu, dW_down, (flags & UNIPOOL_WGRAD_OVERWRITE) != 0};

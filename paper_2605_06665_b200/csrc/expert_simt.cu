@@ -128,13 +128,14 @@ template <typename TE>
 static int wgrad_impl(unipool_ctx* ctx, const PoolWgradArgs& a, cudaStream_t s) {
   const int d = ctx->cfg.d_model, f = ctx->cfg.d_ff;
   // dW_down[e][d, f] += dYp_e^T A_e
-  {
+  if (a.dW_down != nullptr) {
   PhaseTimer pt(ctx, UNIPOOL_PH_WGRAD_DOWN, 1, s);
   grouped_k_gemm_kernel<TE><<<dim3(d / kSimtTile, f / kSimtTile, a.n_experts), kSimtThreads, 0, s>>>(
       static_cast<const TE*>(a.dYp), d, static_cast<const TE*>(a.A), f, a.offsets, a.n_experts,
       a.expert_base, a.n_layers, a.layer_stride_rows, a.dW_down, (int64_t)d * f, d, f, a.overwrite);
   UP_LAUNCH_CHECK();
   }
+  if (a.dW_gu == nullptr) return UNIPOOL_OK;
   PhaseTimer pt(ctx, UNIPOOL_PH_WGRAD_GU, 1, s);
   // dW_gu[e][2f, d] += dGU_e^T Xp_e
   grouped_k_gemm_kernel<TE><<<dim3(2 * f / kSimtTile, d / kSimtTile, a.n_experts), kSimtThreads, 0, s>>>(

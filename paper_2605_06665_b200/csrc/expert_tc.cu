@@ -890,12 +890,14 @@ int wgrad_pair(unipool_ctx* ctx, const PoolWgradArgs& a, cudaStream_t s) {
   p.status = ctx->ws.status;
   CUtensorMap tmP, tmQ, tmW;
   int rc;
-  // dW_down[e] [d, f] (+)= dYp_e^T A_e
-  if ((rc = map_2d(ctx, &tmP, a.dYp, d, rows, 64, 64)) != UNIPOOL_OK) return rc;
-  if ((rc = map_2d(ctx, &tmQ, a.A, f, rows, 64, 64)) != UNIPOOL_OK) return rc;
-  if ((rc = map_chunk(ctx, &tmW, a.dW_down, f, (uint64_t)M * d, kMapF32Chunk)) != UNIPOOL_OK) return rc;
-  p.Mdim = d; p.Ndim = f;
-  if ((rc = launch_wgrad(ctx, UNIPOOL_PH_WGRAD_DOWN, tmP, tmQ, tmW, p, s)) != UNIPOOL_OK) return rc;
+  if (a.dW_down != nullptr) {                     // dW_down[e] [d, f] (+)= dYp_e^T A_e
+    if ((rc = map_2d(ctx, &tmP, a.dYp, d, rows, 64, 64)) != UNIPOOL_OK) return rc;
+    if ((rc = map_2d(ctx, &tmQ, a.A, f, rows, 64, 64)) != UNIPOOL_OK) return rc;
+    if ((rc = map_chunk(ctx, &tmW, a.dW_down, f, (uint64_t)M * d, kMapF32Chunk)) != UNIPOOL_OK) return rc;
+    p.Mdim = d; p.Ndim = f;
+    if ((rc = launch_wgrad(ctx, UNIPOOL_PH_WGRAD_DOWN, tmP, tmQ, tmW, p, s)) != UNIPOOL_OK) return rc;
+  }
+  if (a.dW_gu == nullptr) return UNIPOOL_OK;
   // dW_gu[e] [2f, d] (+)= dGU_e^T Xp_e
   if ((rc = map_2d(ctx, &tmP, a.dGU, 2 * f, rows, 64, 64)) != UNIPOOL_OK) return rc;
   if ((rc = map_2d(ctx, &tmQ, a.Xp, d, rows, 64, 64)) != UNIPOOL_OK) return rc;

@@ -32,3 +32,48 @@ def max_over_ranks(value, world, device="cpu"):
 def whole_job_throughput(units_per_rank, world, ms):
     """Units all ranks processed per second, given the slowest rank's time in milliseconds (weak scaling)."""
     return world * units_per_rank / (ms * 1e-3)
+
+
+class GradientExchange:
+    """The one exchange of a data-parallel training step around the MoE path (the paper's own
+    parallel mode, App. D: data parallel, no expert parallelism): every replica holds the pool and
+    all routers, runs the whole path on its token shard, and the replicas then sum
+
+      * the routing statistics ``counts, score_sum [L, m]`` (before the balance loss, so that the
+        token fractions and mean scores of Eqs. 3-5 are those of the whole batch), and
+      * the fp32 gradients of the pool, the routers and the router scales.
+
+    Reductions are issued asynchronously (``launch``): the collective waits for the work queued so
+    far on the current stream and runs beside what is queued after it, so the pool's dW_down can
+    travel while dW_gu is still being computed; ``finish`` makes the current stream (NCCL) or the
+    host (gloo) wait for all of them.  With one replica every method is the identity.
+    """
+
+    def __init__(self, world, group=None):
+        self.world = int(world)
+        self.group = group
+        self._pending = []
+
+    def global_statistics(self, counts, score_sum):
+        """Sums ``counts`` (int32) and ``score_sum`` (float32) over the replicas in place and returns
+        the factor by which the token count of the balance loss grows (the number of replicas: every
+        replica runs the same number of tokens)."""
+        if self.world > 1:
+            import torch.distributed as dist
+            dist.all_reduce(counts, op=dist.ReduceOp.SUM, group=self.group)
+            dist.all_reduce(score_sum, op=dist.ReduceOp.SUM, group=self.group)
+        return self.world
+
+    def launch(self, tensors):
+        """Starts the sum over replicas of every tensor in ``tensors`` (in place)."""
+        if self.world <= 1:
+            return
+        import torch.distributed as dist
+        for t in tensors:
+            self._pending.append(dist.all_reduce(t, op=dist.ReduceOp.SUM, group=self.group, async_op=True))
+
+    def finish(self):
+        """Returns once every launched reduction is ordered before what the caller does next."""
+        for work in self._pending:
+            work.wait()
+        self._pending = []

@@ -151,8 +151,9 @@ class UniPoolStack:
             self.forward_layer(l, T)
         return self.x[self.L]
 
-    def aux_loss(self, T=None, fbar_prev=None):
-        T = self.T if T is None else T
+    def aux_loss(self, T=None, fbar_prev=None, replicas=1):
+        """``replicas``: the statistics were summed over this many data-parallel replicas of T tokens."""
+        T = (self.T if T is None else T) * replicas
         c = self.ctx
         if fbar_prev is not None and fbar_prev.dim() == 1:
             fbar_prev = fbar_prev.reshape(1, -1)
@@ -184,10 +185,12 @@ class UniPoolStack:
         c.route_bwd(self.x[l], T, self.W_r[l], self.sigma[l], self.m, self.znorm[l], self.z[l],
                     self.idx[l], self.dgate, coef, dx_out, self.dW_r[l], self.dsigma[l:l + 1])
 
-    def backward(self, upstream=None, T=None, with_aux=True, accumulate=True):
+    def backward(self, upstream=None, T=None, with_aux=True, accumulate=True, exchange=None):
         """``accumulate=False``: the pool gradient of this pass replaces the buffers' contents
         (the first weight-gradient contribution to each expert is a store, the rest add), so the
-        buffers need no zeroing; router gradients always add."""
+        buffers need no zeroing; router gradients always add.  ``exchange`` (a
+        ``dp.GradientExchange``): the gradients are summed over the data-parallel replicas, each
+        buffer as soon as it is complete (dW_down while dW_gu is still being computed)."""
         T = self.T if T is None else T
         cur = 0
         if upstream is not None:
@@ -199,18 +202,34 @@ class UniPoolStack:
         if self.deferred_wgrad:
             for g in range(self.G):                        # one pass per sharing group over its layers
                 l0 = g * self.Lg
-                self.ctx.pool_wgrad(self.Lg, self.cap, self.offsets[l0:], self.Xp[l0:], self.A[l0:], self.dYp[l0:],
-                                    self.dGU[l0:], g * self.m, self.m, self.dW_gu, self.dW_down,
-                                    0 if accumulate else B.WGRAD_OVERWRITE)
+                flags = 0 if accumulate else B.WGRAD_OVERWRITE
+                args = (self.Lg, self.cap, self.offsets[l0:], self.Xp[l0:], self.A[l0:], self.dYp[l0:],
+                        self.dGU[l0:], g * self.m, self.m)
+                if exchange is None:
+                    self.ctx.pool_wgrad(*args, self.dW_gu, self.dW_down, flags)
+                else:
+                    e0, e1 = g * self.m, (g + 1) * self.m
+                    self.ctx.pool_wgrad(*args, None, self.dW_down, flags)
+                    exchange.launch([self.dW_down[e0:e1]])
+                    self.ctx.pool_wgrad(*args, self.dW_gu, None, flags)
+                    exchange.launch([self.dW_gu[e0:e1]])
+        if exchange is not None:
+            if not self.deferred_wgrad:
+                exchange.launch([self.dW_down, self.dW_gu])
+            exchange.launch([self.dW_r, self.dsigma])
+            exchange.finish()
         return self.dx[cur]
 
-    def step(self, x0=None, upstream=None, T=None, accumulate=True):
-        """One pass of the whole hot path: forward, balance loss, backward."""
+    def step(self, x0=None, upstream=None, T=None, accumulate=True, exchange=None):
+        """One pass of the whole hot path: forward, balance loss, backward.  With ``exchange`` the
+        step is one data-parallel replica's: the balance loss is taken on the statistics of all
+        replicas' tokens and the gradients are summed over the replicas."""
         self.forward(x0, T)
-        self.aux_loss(T)
+        replicas = 1 if exchange is None else exchange.global_statistics(self.counts, self.score_sum)
+        self.aux_loss(T, replicas=replicas)
         if not accumulate:
             self.zero_router_grad()
-        return self.backward(upstream, T, accumulate=accumulate)
+        return self.backward(upstream, T, accumulate=accumulate, exchange=exchange)
 
     def accumulate_microbatches(self, batches, fbar0=None, T=None):
         """One optimizer step's worth of the path (App. D, App. G): every micro-batch (x0, upstream)

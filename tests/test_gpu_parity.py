@@ -286,6 +286,33 @@ def test_cuda_graph_replay_matches_eager_step():
     st.close()
 
 
+def test_single_replica_exchange_step_is_the_plain_step():
+    """The data-parallel step with one replica (every collective is the identity) issues the weight
+    gradient as two single-product passes: same outputs and gradients as the plain step."""
+    import torch
+    from paper_2605_06665_b200 import dp
+    cfg = small_cfg(dtype="bf16", d=256, f=384, M=16, k=2, L=4, groups=2)
+    T = 700
+    inputs = synth.make_inputs(cfg, seed=10, T=T)
+    x0 = torch.from_numpy(inputs["x0"]).cuda().bfloat16()
+    up = torch.from_numpy(inputs["upstream"]).cuda().bfloat16()
+    for deferred in (True, False):
+        st = build_stack(cfg, inputs, T=T, deferred_wgrad=deferred)
+        st.step(x0, up, accumulate=False)
+        torch.cuda.synchronize()
+        ref = [t.clone() for t in (st.x[cfg["L"]], st.dW_gu, st.dW_down, st.loss, st.dW_r)]
+        for t in (st.dW_gu, st.dW_down):
+            t.fill_(1.0)                               # an overwriting step leaves nothing of this behind
+        st.step(x0, up, accumulate=False, exchange=dp.GradientExchange(1))
+        torch.cuda.synchronize()
+        st.ctx.check_status()
+        got = (st.x[cfg["L"]], st.dW_gu, st.dW_down, st.loss, st.dW_r)
+        for a, b in zip(ref[:4], got[:4]):
+            assert torch.equal(a, b)
+        assert rel_max(to_np(got[4]), to_np(ref[4])) < 1e-5
+        st.close()
+
+
 def test_empty_batch():
     import torch
     cfg = small_cfg()

@@ -397,6 +397,37 @@ def test_sharing_scope_groups_interpolate_between_pool_and_private():
         assert fd(routers2[l]["W_r"], pos) == pytest.approx(res["router_grads"][l]["dW_r"][pos], rel=2e-5, abs=1e-8)
 
 
+def test_data_parallel_replicas_sum_to_the_whole_batch():
+    """Token shards with statistics summed over the replicas: the balance loss is the whole batch's
+    and the replicas' gradients add up to the whole batch's gradient (routing is per token, the
+    objective a sum over tokens plus a loss of batch statistics)."""
+    pool, routers, x0, up, views = tiny_problem(seed=21, L=3, M=6, d=8, f=5, k=2, T=12, bias=True)
+    k, c, eps, alpha = 2, 1.7, 1e-6, 0.3
+    whole = O.stack_objective_and_grads(x0, routers, pool, k, c, eps, alpha, up)
+    shards = [slice(0, 6), slice(6, 12)]
+    local = [O.stack_objective_and_grads(x0[s], routers, pool, k, c, eps, alpha, up[s]) for s in shards]
+    # the layer inputs of a shard are the whole batch's rows: statistics add up exactly
+    counts = sum(r["counts"] for r in local)
+    S = sum(r["S"] for r in local)
+    assert (counts == whole["counts"]).all()
+    np.testing.assert_allclose(S, whole["S"], rtol=1e-13)
+    reps = [O.stack_objective_and_grads(x0[s], routers, pool, k, c, eps, alpha, up[s],
+                                        replica_stats=lambda cn, ss: (counts, S, 12)) for s in shards]
+    for r in reps:
+        assert r["loss_aux"] == pytest.approx(whole["loss_aux"], rel=1e-13)
+    # without the summed statistics the shards' losses do NOT average to the whole batch's
+    assert abs(0.5 * (local[0]["loss_aux"] + local[1]["loss_aux"]) - whole["loss_aux"]) > 1e-6
+    for name in ("W_gate", "W_up", "W_down"):
+        np.testing.assert_allclose(reps[0]["pool_grad"][name] + reps[1]["pool_grad"][name],
+                                   whole["pool_grad"][name], rtol=1e-10, atol=1e-13)
+    for l in range(3):
+        np.testing.assert_allclose(reps[0]["router_grads"][l]["dW_r"] + reps[1]["router_grads"][l]["dW_r"],
+                                   whole["router_grads"][l]["dW_r"], rtol=1e-10, atol=1e-13)
+        assert reps[0]["router_grads"][l]["dsigma"] + reps[1]["router_grads"][l]["dsigma"] == pytest.approx(
+            whole["router_grads"][l]["dsigma"], rel=1e-10)
+    np.testing.assert_allclose(np.concatenate([r["dx0"] for r in reps]), whole["dx0"], rtol=1e-10, atol=1e-13)
+
+
 def test_unique_expert_accounting():
     """App. E: private experts give U = L exactly for top-1 (L k for top-k); a shared pool gives
     1 <= U <= min(M, L k); a hand case; and U equals the row-wise count of a dense indicator matrix."""
