@@ -48,6 +48,7 @@ enum Mode : int {
 struct GemmParams {
   const int32_t* offsets;       // row tiles: &offsets[n_experts]; wgrad: [n_layers][n_experts+1]
   const int32_t* tile_expert;   // row tiles only
+  const int32_t* group_offsets; // row tiles on CTA pairs: [n_experts + 1] starts of the groups
   int n_experts, expert_base;
   int n_layers;                 // wgrad
   int layer_stride_rows;        // wgrad
@@ -201,6 +202,72 @@ struct ChunkCursor {
   }
   __device__ int col() const { return nt * BN + ch * kChunk; }
 };
+
+// Epilogue of the gate/up projection for one warp's 32 rows: G and U leave TMEM, A = silu(G) * U is
+// formed, and the three bf16 chunks are staged and stored (GU through tmC0, A through tmC1).
+// Warps that share a TMEM lane quarter split the chunks: this warp takes ch0, ch0 + step, ...
+__device__ __forceinline__ void epilogue_swiglu(const CUtensorMap* tmC0, const CUtensorMap* tmC1, const GemmParams& p,
+                                                uint32_t t_row, int nt, int row0, uint8_t* stg, int lane,
+                                                int ch0 = 0, int step = 1) {
+#pragma unroll 1
+  for (int ch = ch0; ch < BN / 2 / kChunk; ch += step) {
+    const int feat = nt * (BN / 2) + ch * kChunk;
+    if (feat >= p.f) break;
+    uint32_t rg[32], ru[32];
+    tc::tmem_ld_32x32(t_row + ch * kChunk, rg);
+    tc::tmem_ld_32x32(t_row + BN / 2 + ch * kChunk, ru);
+    tc::tmem_ld_wait();
+    float g[32], u[32], a[32];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      g[i] = __uint_as_float(rg[i]);
+      u[i] = __uint_as_float(ru[i]);
+      a[i] = g[i] * sigmoid_fast(g[i]) * u[i];
+    }
+    // lanes 0, 1, 2 each own one of the three stores (G, U, A), so the stores are issued and
+    // their shared-memory reads awaited side by side
+    if (lane < 3) tc::bulk_wait_read<0>();       // the previous chunk's stores have drained the tiles
+    __syncwarp();
+    stage_row_bf16(stg, lane, g);
+    stage_row_bf16(stg + kBf16ChunkBytes, lane, u);
+    stage_row_bf16(stg + 2 * kBf16ChunkBytes, lane, a);
+    tc::fence_proxy_async();
+    __syncwarp();
+    if (lane == 0) tc::tma_store_2d(tmC0, stg, feat, row0);
+    else if (lane == 1) tc::tma_store_2d(tmC0, stg + kBf16ChunkBytes, p.f + feat, row0);
+    else if (lane == 2) tc::tma_store_2d(tmC1, stg + 2 * kBf16ChunkBytes, feat, row0);
+    if (lane < 3) tc::bulk_commit();
+  }
+}
+
+// Epilogue of a plain row-tile GEMM (down projection, second dgrad) for one warp's 32 rows: the
+// accumulator is rounded to bf16, staged in a ring of four chunk tiles and stored (or add-reduced).
+template <int MODE>
+__device__ __forceinline__ void epilogue_rows(const CUtensorMap* tmC0, const GemmParams& p, uint32_t t_row, int nt,
+                                              int row0, uint8_t* stg, int lane, int& gchunk, int ch0 = 0, int step = 1) {
+#pragma unroll 1
+  for (int ch = ch0; ch < BN / kChunk; ch += step) {
+    const int col = nt * BN + ch * kChunk;
+    if (col >= p.Ndim) break;
+    uint32_t rr[32];
+    tc::tmem_ld_32x32(t_row + ch * kChunk, rr);
+    tc::tmem_ld_wait();
+    float v[32];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(rr[i]);
+    uint8_t* buf = stg + (gchunk++ & 3) * kBf16ChunkBytes;
+    if (lane == 0) tc::bulk_wait_read<3>();      // the store issued four chunks ago has drained `buf`
+    __syncwarp();
+    stage_row_bf16(buf, lane, v);
+    tc::fence_proxy_async();
+    __syncwarp();
+    if (lane == 0) {
+      if (MODE == kFwd2 || p.overwrite) tc::tma_store_2d(tmC0, buf, col, row0);
+      else tc::tma_reduce_add_2d(tmC0, buf, col, row0);
+      tc::bulk_commit();
+    }
+  }
+}
 
 template <int MODE>
 __global__ void __launch_bounds__(Traits<MODE>::kThreads, 1)
@@ -447,58 +514,9 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
       const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * BN;
 
       if constexpr (MODE == kFwd1) {
-#pragma unroll 1
-        for (int ch = 0; ch < BN / 2 / kChunk; ++ch) {
-          const int feat = c.nt * (BN / 2) + ch * kChunk;
-          if (feat >= p.f) break;
-          uint32_t rg[32], ru[32];
-          tc::tmem_ld_32x32(t_row + ch * kChunk, rg);
-          tc::tmem_ld_32x32(t_row + BN / 2 + ch * kChunk, ru);
-          tc::tmem_ld_wait();
-          float g[32], u[32], a[32];
-#pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            g[i] = __uint_as_float(rg[i]);
-            u[i] = __uint_as_float(ru[i]);
-            a[i] = g[i] * sigmoid_fast(g[i]) * u[i];
-          }
-          // lanes 0, 1, 2 each own one of the three stores (G, U, A), so the stores are issued and
-          // their shared-memory reads awaited side by side
-          if (lane < 3) tc::bulk_wait_read<0>();       // the previous chunk's stores have drained the tiles
-          __syncwarp();
-          stage_row_bf16(stg, lane, g);
-          stage_row_bf16(stg + kBf16ChunkBytes, lane, u);
-          stage_row_bf16(stg + 2 * kBf16ChunkBytes, lane, a);
-          tc::fence_proxy_async();
-          __syncwarp();
-          if (lane == 0) tc::tma_store_2d(&tmC0, stg, feat, row0);
-          else if (lane == 1) tc::tma_store_2d(&tmC0, stg + kBf16ChunkBytes, p.f + feat, row0);
-          else if (lane == 2) tc::tma_store_2d(&tmC1, stg + 2 * kBf16ChunkBytes, feat, row0);
-          if (lane < 3) tc::bulk_commit();
-        }
+        epilogue_swiglu(&tmC0, &tmC1, p, t_row, c.nt, row0, stg, lane);
       } else if constexpr (MODE == kFwd2 || MODE == kDgrad2) {
-#pragma unroll 1
-        for (int ch = 0; ch < BN / kChunk; ++ch) {
-          const int col = c.nt * BN + ch * kChunk;
-          if (col >= p.Ndim) break;
-          uint32_t rr[32];
-          tc::tmem_ld_32x32(t_row + ch * kChunk, rr);
-          tc::tmem_ld_wait();
-          float v[32];
-#pragma unroll
-          for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(rr[i]);
-          uint8_t* buf = stg + (gchunk++ & 3) * kBf16ChunkBytes;
-          if (lane == 0) tc::bulk_wait_read<3>();      // the store issued four chunks ago has drained `buf`
-          __syncwarp();
-          stage_row_bf16(buf, lane, v);
-          tc::fence_proxy_async();
-          __syncwarp();
-          if (lane == 0) {
-            if (MODE == kFwd2 || p.overwrite) tc::tma_store_2d(&tmC0, buf, col, row0);
-            else tc::tma_reduce_add_2d(&tmC0, buf, col, row0);
-            tc::bulk_commit();
-          }
-        }
+        epilogue_rows<MODE>(&tmC0, p, t_row, c.nt, row0, stg, lane, gchunk);
       } else if constexpr (MODE == kDgrad1) {
 #pragma unroll 1
         for (int ch = 0; ch < nch; ++ch) {
@@ -586,7 +604,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
 // even CTA issues the MMAs; every TMA load counts its bytes on the even CTA's mbarrier (plain
 // loads, no multicast); tcgen05.commit arrives on the stage / accumulator barriers of both CTAs.
 constexpr int kPairStages = 6;
-constexpr uint32_t kPairSmemTotal = kSmemTotal + UNIPOOL_MAX_EXPERTS * sizeof(uint16_t);   // + the experts' order
+constexpr uint32_t kPairSmemTotal = kSmemTotal + (UNIPOOL_MAX_EXPERTS + 8) * sizeof(uint16_t);   // + one entry per expert
 static_assert(kPairSmemTotal <= 227 * 1024, "shared-memory budget");
 constexpr uint32_t kPairHalfBytes = 128 * BK * 2;            // 128 (M or N) x 64 (K) bf16
 constexpr uint32_t kPairStageBytes = 2 * kPairHalfBytes;
@@ -853,6 +871,209 @@ int map_chunk(const unipool_ctx* ctx, CUtensorMap* out, const void* base, uint64
   return map_2d(ctx, out, base, cols, rows, kChunk, 32, kind);
 }
 
+// ---------------------------------------------------------------- row-tile GEMMs on CTA pairs
+// The forward GEMMs and the second dgrad at small groups are bound by what the SMs can pull in: a
+// 128 x 256 tile takes 48 KB of operands per k-block, most of it the expert's weights, which the
+// other row tiles of the same expert fetch again.  Here two row tiles of ONE expert share a CTA pair:
+// one tcgen05.mma.cta_group::2 of M = 256 (128 rows per CTA, each in its own TMEM) and N = 256, each
+// CTA loading its own 128 rows of A and HALF of the expert's 256 weight rows (B), 32 KB per k-block
+// and CTA, six stages.  A group with an odd number of row tiles ends in a pair whose second CTA has
+// no rows: it still supplies its half of B, loads no A, and stores nothing.  Scheduling, barriers and
+// commits follow the weight-gradient pair kernel above; the epilogues are the single-CTA ones.
+// Six operand stages and four epilogue warps: a variant with eight epilogue warps (two per TMEM lane
+// quarter, taking alternate chunks; the helpers below support it) had to give one stage to their
+// staging tiles and was 8 - 12 % slower - the main loop lives on the bytes it keeps in flight.
+constexpr int kRowPairStages = 6;
+constexpr int kRowPairEpiWarps = 4;
+constexpr int kRowPairThreads = 64 + 32 * kRowPairEpiWarps;
+static_assert(kRowPairStages * kPairStageBytes + kRowPairEpiWarps * 8192 == kBarOffset, "shared-memory budget");
+
+struct PairTile { int e, mt, nt; bool mine, peer; };
+
+// pair-tile q of the row space -> expert and first row tile; pp[e] = pair-tiles before expert e
+__device__ __forceinline__ PairTile pair_tile(const GemmParams& p, const uint16_t* pp, int tile, int n_nt,
+                                              int total_q, bool descending, int rank) {
+  PairTile t;
+  int q = tile / n_nt;
+  t.nt = tile % n_nt;
+  if (descending) q = total_q - 1 - q;
+  int lo = 0, hi = p.n_experts - 1;                    // last e with pp[e] <= q
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if ((int)pp[mid] <= q) lo = mid; else hi = mid - 1;
+  }
+  t.e = lo;
+  const int first = p.group_offsets[lo] / BM, n_tiles = (p.group_offsets[lo + 1] - p.group_offsets[lo]) / BM;
+  const int i = 2 * (q - (int)pp[lo]);
+  t.mt = first + i + rank;
+  t.mine = i + rank < n_tiles;
+  t.peer = i + (rank ^ 1) < n_tiles;
+  return t;
+}
+
+template <int MODE>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kRowPairThreads, 1)
+row_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                const __grid_constant__ CUtensorMap tmC0, const __grid_constant__ CUtensorMap tmC1,
+                const GemmParams p) {
+  static_assert(MODE == kFwd1 || MODE == kFwd2 || MODE == kDgrad2, "row tiles without epilogue operands");
+  constexpr bool kBMn = Traits<MODE>::kBMn;
+  constexpr bool kDescending = MODE == kFwd2 || MODE == kDgrad2;      // see tile_coord
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + kBarOffset);
+  uint64_t* empty_bar = full_bar + kRowPairStages;
+  uint64_t* tmem_full = empty_bar + kRowPairStages;
+  uint64_t* tmem_empty = tmem_full + 2;
+  uint32_t* tmem_ptr = reinterpret_cast<uint32_t*>(tmem_empty + 2);
+  volatile int* abort = reinterpret_cast<volatile int*>(tmem_ptr + 1);
+  uint16_t* pp = reinterpret_cast<uint16_t*>(smem + kBarOffset + 512);       // [n_experts + 1]
+
+  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+  const int rank = (int)tc::cluster_ctarank();               // 0 = leader
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kRowPairStages; ++s) { tc::mbar_init(&full_bar[s], 1); tc::mbar_init(&empty_bar[s], 1); }
+    for (int a = 0; a < 2; ++a) { tc::mbar_init(&tmem_full[a], 1); tc::mbar_init(&tmem_empty[a], 2 * kRowPairEpiWarps); }
+    *abort = 0;
+    tc::fence_barrier_init();
+    tc::tma_prefetch_desc(&tmA);
+    tc::tma_prefetch_desc(&tmB);
+    tc::tma_prefetch_desc(&tmC0);
+    if constexpr (MODE == kFwd1) tc::tma_prefetch_desc(&tmC1);
+  }
+  if (warp == 1) {
+    tc::tmem_alloc_pair(tmem_ptr, 512);
+    tc::tmem_relinquish_pair();
+  }
+  // pair-tiles before each expert: an expert of n row tiles takes ceil(n / 2)
+  for (int e = threadIdx.x; e <= p.n_experts; e += blockDim.x) {
+    int before = 0;
+    for (int o = 0; o < e; ++o) before += ((p.group_offsets[o + 1] - p.group_offsets[o]) / BM + 1) >> 1;
+    pp[e] = (uint16_t)before;
+  }
+  tc::tc_fence_before_sync();
+  __syncthreads();
+  tc::cluster_sync();                                        // both CTAs' barriers exist before any remote use
+  tc::tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_ptr;
+
+  const int ncols = MODE == kFwd1 ? BN / 2 : BN;             // output columns (fwd1: features) per tile
+  const int n_nt = (p.Ndim + ncols - 1) / ncols;
+  const int total_q = pp[p.n_experts];
+  const int total = total_q * n_nt;
+  const int kblocks = p.Kdim / BK;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer (one in each CTA)
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = pair; tile < total && ok; tile += n_pairs) {
+        const PairTile t = pair_tile(p, pp, tile, n_nt, total_q, kDescending, rank);
+        const int pe = p.expert_base + t.e;
+        const uint32_t tx = 2 * kPairHalfBytes + (t.mine ? kPairHalfBytes : 0) + (t.peer ? kPairHalfBytes : 0);
+        for (int kb = 0; kb < kblocks; ++kb) {
+          if (!tc::mbar_wait(&empty_bar[stage], phase ^ 1u, abort)) { report_timeout(p, abort, 31); ok = false; break; }
+          uint8_t* sA = smem + stage * kPairStageBytes;
+          uint8_t* sB = sA + kPairHalfBytes;
+          if (rank == 0) tc::mbar_expect_tx(&full_bar[stage], tx);              // both CTAs' bytes
+          if (t.mine) tc::tma_load_2d_pair(sA, &tmA, &full_bar[stage], kb * BK, t.mt * BM);
+          if constexpr (MODE == kFwd1) {           // B rows: 128 gate features (leader) or the same 128 up features
+            tc::tma_load_2d_pair(sB, &tmB, &full_bar[stage], kb * BK, pe * 2 * p.f + rank * p.f + t.nt * (BN / 2));
+          } else if constexpr (MODE == kFwd2) {
+            tc::tma_load_2d_pair(sB, &tmB, &full_bar[stage], kb * BK, pe * p.Ndim + t.nt * BN + rank * (BN / 2));
+          } else {
+#pragma unroll
+            for (int i = 0; i < 2; ++i)
+              tc::tma_load_2d_pair(sB + i * kMnBlockBytes, &tmB, &full_bar[stage],
+                                   t.nt * BN + rank * (BN / 2) + 64 * i, pe * p.Kdim + kb * BK);
+          }
+          if (++stage == kRowPairStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok)
+        for (int i = 0; i < 200; ++i) __nanosleep(1000);
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer (leader CTA only)
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = tc::instr_desc_bf16(BN, false, kBMn, 256);
+      constexpr uint32_t b_lbo = kBMn ? kMnBlockBytes : 16;
+      constexpr uint32_t a_step = 32 >> 4;                                   // K-major: 32 bytes per K = 16
+      constexpr uint32_t b_step = (kBMn ? 16 * 128 : 32) >> 4;
+      int stage = 0;
+      uint32_t phase = 0;
+      int local = 0;
+      bool ok = true;
+      for (int tile = pair; tile < total && ok; tile += n_pairs) {
+        const int acc = local & 1;
+        const uint32_t acc_phase = (local >> 1) & 1;
+        ++local;
+        if (!tc::mbar_wait(&tmem_empty[acc], acc_phase ^ 1u, abort)) { report_timeout(p, abort, 32); break; }
+        tc::tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + acc * BN;
+        for (int kb = 0; kb < kblocks; ++kb) {
+          if (!tc::mbar_wait(&full_bar[stage], phase, abort)) { report_timeout(p, abort, 33); ok = false; break; }
+          tc::tc_fence_after_sync();
+          const uint32_t aaddr = tc::smem_u32(smem + stage * kPairStageBytes);
+          const uint64_t adesc = tc::smem_desc_sw128(aaddr, 16, 1024);
+          const uint64_t bdesc = tc::smem_desc_sw128(aaddr + kPairHalfBytes, b_lbo, 1024);
+#pragma unroll
+          for (int j = 0; j < BK / 16; ++j)
+            tc::umma_bf16_pair(d_tmem, adesc + j * a_step, bdesc + j * b_step, idesc, (kb | j) != 0 ? 1u : 0u);
+          tc::umma_commit_pair(&empty_bar[stage], 3);           // frees the stage in both CTAs
+          if (++stage == kRowPairStages) { stage = 0; phase ^= 1u; }
+        }
+        if (ok) tc::umma_commit_pair(&tmem_full[acc], 3);       // accumulator complete, both CTAs
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue: this CTA's row tile
+    const int quarter = warp & 3;
+    const int half = (warp - 2) >> 2;                    // which of the quarter's two warps
+    uint8_t* stg = smem + kRowPairStages * kPairStageBytes + (warp - 2) * 8192;
+    int gchunk = 0, local = 0;
+    (void)gchunk;
+    for (int tile = pair; tile < total; tile += n_pairs) {
+      const PairTile t = pair_tile(p, pp, tile, n_nt, total_q, kDescending, rank);
+      const int acc = local & 1;
+      const uint32_t acc_phase = (local >> 1) & 1;
+      ++local;
+      if (!tc::mbar_wait(&tmem_full[acc], acc_phase, abort)) {
+        if (lane == 0) report_timeout(p, abort, 34);
+        break;
+      }
+      tc::tc_fence_after_sync();
+      if (t.mine) {
+        const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * BN;
+        const int row0 = t.mt * BM + quarter * 32;
+        constexpr int kShare = kRowPairEpiWarps / 4;     // warps per TMEM lane quarter
+        if constexpr (MODE == kFwd1) epilogue_swiglu(&tmC0, &tmC1, p, t_row, t.nt, row0, stg, lane, half, kShare);
+        else epilogue_rows<MODE>(&tmC0, p, t_row, t.nt, row0, stg, lane, gchunk, half, kShare);
+      }
+      tc::tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) {                                   // the leader's MMA thread waits for both CTAs' epilogue warps
+        if (rank == 0) tc::mbar_arrive(&tmem_empty[acc]);
+        else tc::mbar_arrive_leader(&tmem_empty[acc]);
+      }
+    }
+    if (lane < 3) tc::bulk_wait<0>();
+    __syncwarp();
+  }
+
+  tc::tc_fence_before_sync();
+  __syncthreads();
+  tc::cluster_sync();                                        // neither CTA leaves while the other may still signal it
+  if (warp == 1) {
+    tc::tc_fence_after_sync();
+    tc::tmem_dealloc_pair(tmem_base, 512);
+  }
+}
+
 template <int MODE>
 int launch(unipool_ctx* ctx, int phase, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC0,
            const CUtensorMap& tmC1, const GemmParams& p, cudaStream_t s) {
@@ -860,6 +1081,29 @@ int launch(unipool_ctx* ctx, int phase, const CUtensorMap& tmA, const CUtensorMa
   auto kern = grouped_gemm_tc_kernel<MODE>;
   UP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemTotal));
   kern<<<ctx->sm_count, Traits<MODE>::kThreads, kSmemTotal, s>>>(tmA, tmB, tmC0, tmC1, p);
+  UP_LAUNCH_CHECK();
+  return UNIPOOL_OK;
+}
+
+// Row-tile GEMMs run on CTA pairs (UNIPOOL_ROW_PAIR=0, a debugging aid, selects the single-CTA
+// kernel); the pair schedule keeps 16-bit counts of pair-tiles.
+// A group of an odd number of row tiles wastes half of its last pair, so pairs pay once groups are
+// several tiles long: they are used when a batch of max_tokens gives the average expert at least
+// four row tiles (UNIPOOL_ROW_PAIR=1 forces them on, =0 off).
+bool rows_on_pairs(const unipool_ctx* ctx, int n_experts) {
+  static const int forced = [] { const char* v = getenv("UNIPOOL_ROW_PAIR"); return v ? (v[0] == '0' ? 0 : 1) : -1; }();
+  if (ctx->sm_count < 2 || ctx->row_capacity / (2 * BM) + n_experts >= 65535) return false;
+  if (forced >= 0) return forced == 1;
+  return (int64_t)ctx->cfg.max_tokens * ctx->cfg.top_k >= (int64_t)4 * BM * n_experts;
+}
+
+template <int MODE>
+int launch_row_pairs(unipool_ctx* ctx, int phase, const CUtensorMap& tmA, const CUtensorMap& tmB,
+                     const CUtensorMap& tmC0, const CUtensorMap& tmC1, const GemmParams& p, cudaStream_t s) {
+  PhaseTimer pt(ctx, phase, 1, s);
+  auto kern = row_pair_kernel<MODE>;
+  UP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPairSmemTotal));
+  kern<<<ctx->sm_count / 2 * 2, kRowPairThreads, kPairSmemTotal, s>>>(tmA, tmB, tmC0, tmC1, p);
   UP_LAUNCH_CHECK();
   return UNIPOOL_OK;
 }
@@ -934,12 +1178,17 @@ int expert_fwd_tc(unipool_ctx* ctx, const ExpertFwdArgs& a, cudaStream_t s) {
   p.expert_base = a.expert_base;
   p.f = f;
   p.status = ctx->ws.status;
+  p.group_offsets = a.offsets;
+  const bool pairs = rows_on_pairs(ctx, a.n_experts);
   CUtensorMap tmA, tmB, tmC0, tmC1;
   int rc;
   // GU = Xp [W_gate; W_up]^T with the SwiGLU epilogue.  B tile = 128 gate rows + 128 up rows of the
-  // same features, fetched as one 3-D box over W_gu viewed as [2M, f, d].
+  // same features, fetched as one 3-D box over W_gu viewed as [2M, f, d] (CTA pairs: one half each,
+  // 128 rows of W_gu viewed as [2M f, d]).
   if ((rc = map_2d(ctx, &tmA, a.Xp, d, cap, 64, BM)) != UNIPOOL_OK) return rc;
-  {
+  if (pairs) {
+    if ((rc = map_2d(ctx, &tmB, a.W_gu, d, (uint64_t)M * 2 * f, 64, BN / 2)) != UNIPOOL_OK) return rc;
+  } else {
     const uint64_t dims[3] = {(uint64_t)d, (uint64_t)f, (uint64_t)2 * M};
     const uint64_t strides[2] = {(uint64_t)d, (uint64_t)f * d};
     const uint32_t box[3] = {64, BN / 2, 2};
@@ -948,13 +1197,16 @@ int expert_fwd_tc(unipool_ctx* ctx, const ExpertFwdArgs& a, cudaStream_t s) {
   if ((rc = map_chunk(ctx, &tmC0, a.GU, 2 * f, cap, kMapBf16Chunk)) != UNIPOOL_OK) return rc;
   if ((rc = map_chunk(ctx, &tmC1, a.A, f, cap, kMapBf16Chunk)) != UNIPOOL_OK) return rc;
   p.Ndim = f; p.Kdim = d;
-  if ((rc = launch<kFwd1>(ctx, UNIPOOL_PH_EXPERT_FWD_GU, tmA, tmB, tmC0, tmC1, p, s)) != UNIPOOL_OK) return rc;
+  rc = pairs ? launch_row_pairs<kFwd1>(ctx, UNIPOOL_PH_EXPERT_FWD_GU, tmA, tmB, tmC0, tmC1, p, s)
+             : launch<kFwd1>(ctx, UNIPOOL_PH_EXPERT_FWD_GU, tmA, tmB, tmC0, tmC1, p, s);
+  if (rc != UNIPOOL_OK) return rc;
   // Yp = A W_down^T
   if ((rc = map_2d(ctx, &tmA, a.A, f, cap, 64, BM)) != UNIPOOL_OK) return rc;
-  if ((rc = map_2d(ctx, &tmB, a.W_down, f, (uint64_t)M * d, 64, BN)) != UNIPOOL_OK) return rc;
+  if ((rc = map_2d(ctx, &tmB, a.W_down, f, (uint64_t)M * d, 64, pairs ? BN / 2 : BN)) != UNIPOOL_OK) return rc;
   if ((rc = map_chunk(ctx, &tmC0, a.Yp, d, cap, kMapBf16Chunk)) != UNIPOOL_OK) return rc;
   p.Ndim = d; p.Kdim = f;
-  return launch<kFwd2>(ctx, UNIPOOL_PH_EXPERT_FWD_DOWN, tmA, tmB, tmC0, tmC0, p, s);
+  return pairs ? launch_row_pairs<kFwd2>(ctx, UNIPOOL_PH_EXPERT_FWD_DOWN, tmA, tmB, tmC0, tmC0, p, s)
+               : launch<kFwd2>(ctx, UNIPOOL_PH_EXPERT_FWD_DOWN, tmA, tmB, tmC0, tmC0, p, s);
 }
 
 int expert_bwd_tc(unipool_ctx* ctx, const ExpertBwdArgs& a, cudaStream_t s) {
@@ -981,7 +1233,10 @@ int expert_bwd_tc(unipool_ctx* ctx, const ExpertBwdArgs& a, cudaStream_t s) {
   if ((rc = map_2d(ctx, &tmB, a.W_gu, d, (uint64_t)M * 2 * f, 64, 64)) != UNIPOOL_OK) return rc;
   if ((rc = map_chunk(ctx, &tmC0, a.dXp, d, cap, kMapBf16Chunk)) != UNIPOOL_OK) return rc;
   p.Ndim = d; p.Kdim = 2 * f; p.overwrite = 1;
-  if ((rc = launch<kDgrad2>(ctx, UNIPOOL_PH_DGRAD_GU, tmA, tmB, tmC0, tmC0, p, s)) != UNIPOOL_OK) return rc;
+  p.group_offsets = a.offsets;
+  rc = rows_on_pairs(ctx, a.n_experts) ? launch_row_pairs<kDgrad2>(ctx, UNIPOOL_PH_DGRAD_GU, tmA, tmB, tmC0, tmC0, p, s)
+                                       : launch<kDgrad2>(ctx, UNIPOOL_PH_DGRAD_GU, tmA, tmB, tmC0, tmC0, p, s);
+  if (rc != UNIPOOL_OK) return rc;
   if (a.wgrad) {
     PoolWgradArgs w{1, 0, a.offsets, a.Xp, a.A, a.dYp, a.dGU, a.expert_base, a.n_experts, a.dW_gu, a.dW_down,
                     a.overwrite};
