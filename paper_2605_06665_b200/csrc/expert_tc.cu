@@ -1087,14 +1087,15 @@ int launch(unipool_ctx* ctx, int phase, const CUtensorMap& tmA, const CUtensorMa
 
 // Row-tile GEMMs run on CTA pairs (UNIPOOL_ROW_PAIR=0, a debugging aid, selects the single-CTA
 // kernel); the pair schedule keeps 16-bit counts of pair-tiles.
-// A group of an odd number of row tiles wastes half of its last pair, so pairs pay once groups are
-// several tiles long: they are used when a batch of max_tokens gives the average expert at least
-// four row tiles (UNIPOOL_ROW_PAIR=1 forces them on, =0 off).
+// A group of an odd number of row tiles wastes half of its last pair (tensor work and power), so
+// pairs pay once groups are many tiles long: measured neutral to slightly worse at 3 - 7 tiles per
+// group, 10 % faster per GEMM at 32.  They are used when a batch of max_tokens gives the average
+// expert at least eight row tiles (UNIPOOL_ROW_PAIR=1 forces them on, =0 off).
 bool rows_on_pairs(const unipool_ctx* ctx, int n_experts) {
   static const int forced = [] { const char* v = getenv("UNIPOOL_ROW_PAIR"); return v ? (v[0] == '0' ? 0 : 1) : -1; }();
   if (ctx->sm_count < 2 || ctx->row_capacity / (2 * BM) + n_experts >= 65535) return false;
   if (forced >= 0) return forced == 1;
-  return (int64_t)ctx->cfg.max_tokens * ctx->cfg.top_k >= (int64_t)4 * BM * n_experts;
+  return (int64_t)ctx->cfg.max_tokens * ctx->cfg.top_k >= (int64_t)8 * BM * n_experts;
 }
 
 template <int MODE>
