@@ -186,19 +186,18 @@ def run_ours(args):
         st.step(x0, up, accumulate=False, exchange=exchange)
 
     def e2e_step():
-        st.step(x0_host, up_host, accumulate=False, exchange=exchange)   # H2D copies of this step's inputs from pinned memory
-        xL_host.copy_(st.x[L], non_blocking=True)
+        # H2D copies of this step's inputs from pinned memory, D2H of x_L (beside the compute) and of the loss
+        st.step(x0_host, up_host, accumulate=False, exchange=exchange, out=xL_host)
         loss_host.copy_(st.loss, non_blocking=True)
 
     if args.graph:                           # one CUDA graph per step variant: same kernels, one launch
         g_dev = st.capture_step(x0, up, accumulate=False)
-        g_e2e = st.capture_step(x0_host, up_host, accumulate=False)
+        g_e2e = st.capture_step(x0_host, up_host, accumulate=False, out=xL_host)
         eager_step = device_step
         device_step = g_dev.replay
 
         def e2e_step():
             g_e2e.replay()
-            xL_host.copy_(st.x[L], non_blocking=True)
             loss_host.copy_(st.loss, non_blocking=True)
     else:
         eager_step = device_step

@@ -95,6 +95,7 @@ class UniPoolStack:
         self.coef = e(n_aux, self.m, dtype=f32)
         self.fbar = e(n_aux, self.m, dtype=f32)
         self.fbar_lag = None                               # f-bar of the previous micro-batch (App. G)
+        self._copy_stream = None                           # host <-> device copies beside the compute
 
     # ------------------------------------------------------------------ parameters
     def load(self, pool, routers):
@@ -220,16 +221,43 @@ class UniPoolStack:
             exchange.finish()
         return self.dx[cur]
 
-    def step(self, x0=None, upstream=None, T=None, accumulate=True, exchange=None):
+    def step(self, x0=None, upstream=None, T=None, accumulate=True, exchange=None, out=None):
         """One pass of the whole hot path: forward, balance loss, backward.  With ``exchange`` the
         step is one data-parallel replica's: the balance loss is taken on the statistics of all
-        replicas' tokens and the gradients are summed over the replicas."""
+        replicas' tokens and the gradients are summed over the replicas.
+        Host-resident tensors (pinned memory) are moved beside the compute on a second stream: an
+        ``upstream`` on the host is copied in while the forward pass runs, and ``out`` (host or
+        device, [T, d]) receives x_L while the backward pass runs; both copies are ordered before
+        the step's end on the calling stream."""
+        T_ = self.T if T is None else T
+        cur = torch.cuda.current_stream(self.device)
+        side = None
+        up_ready = None
+        if (upstream is not None and not upstream.is_cuda) or out is not None:
+            if self._copy_stream is None:
+                self._copy_stream = torch.cuda.Stream(self.device)
+            side = self._copy_stream
+            side.wait_stream(cur)                          # nothing queued before this step still uses dx / out
+        if upstream is not None and not upstream.is_cuda:
+            with torch.cuda.stream(side):
+                self.dx[0, :T_].copy_(upstream, non_blocking=True)
+                up_ready = side.record_event()
+            upstream = None                                # backward starts from dx[0]
         self.forward(x0, T)
+        if out is not None:
+            side.wait_stream(cur)
+            with torch.cuda.stream(side):
+                out.copy_(self.x[self.L, :T_], non_blocking=True)
         replicas = 1 if exchange is None else exchange.global_statistics(self.counts, self.score_sum)
         self.aux_loss(T, replicas=replicas)
         if not accumulate:
             self.zero_router_grad()
-        return self.backward(upstream, T, accumulate=accumulate, exchange=exchange)
+        if up_ready is not None:
+            cur.wait_event(up_ready)
+        dx0 = self.backward(upstream, T, accumulate=accumulate, exchange=exchange)
+        if side is not None:
+            cur.wait_stream(side)
+        return dx0
 
     def accumulate_microbatches(self, batches, fbar0=None, T=None):
         """One optimizer step's worth of the path (App. D, App. G): every micro-batch (x0, upstream)
@@ -251,7 +279,7 @@ class UniPoolStack:
             self.backward(upstream, T, accumulate=i > 0)
         return losses
 
-    def capture_step(self, x0=None, upstream=None, accumulate=True):
+    def capture_step(self, x0=None, upstream=None, accumulate=True, out=None):
         """Records one whole step (the library calls of ``step`` with these tensors) into a CUDA graph
         and returns it; ``graph.replay()`` then issues the step with one launch.  Every call of the
         path is asynchronous on the stream and allocates nothing, so the recording holds exactly the
@@ -259,11 +287,11 @@ class UniPoolStack:
         side = torch.cuda.Stream(self.device)
         side.wait_stream(torch.cuda.current_stream(self.device))
         with torch.cuda.stream(side):                       # one eager pass first: lazy set-up happens here
-            self.step(x0, upstream, accumulate=accumulate)
+            self.step(x0, upstream, accumulate=accumulate, out=out)
         torch.cuda.current_stream(self.device).wait_stream(side)
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph, stream=side):
-            self.step(x0, upstream, accumulate=accumulate)
+            self.step(x0, upstream, accumulate=accumulate, out=out)
         return graph
 
     def close(self):

@@ -317,6 +317,40 @@ def test_single_replica_exchange_step_is_the_plain_step():
         st.close()
 
 
+def test_host_resident_step_matches_device_resident_step():
+    """Inputs in pinned host memory (upstream copied in during the forward pass, x_L copied out during
+    the backward pass, on a second stream) give the same step, eagerly and from a CUDA graph."""
+    import torch
+    cfg = small_cfg(dtype="bf16", d=256, f=384, M=16, k=2, L=3)
+    T = 900
+    inputs = synth.make_inputs(cfg, seed=12, T=T)
+    x0_h = torch.from_numpy(inputs["x0"]).bfloat16().pin_memory()
+    up_h = torch.from_numpy(inputs["upstream"]).bfloat16().pin_memory()
+    out_h = torch.zeros_like(x0_h).pin_memory()
+    st = build_stack(cfg, inputs, T=T, deferred_wgrad=True)
+    dx_ref = st.step(x0_h.cuda(), up_h.cuda(), accumulate=False).clone()
+    torch.cuda.synchronize()
+    ref = [t.clone() for t in (st.x[cfg["L"]], st.dW_gu, st.dW_down)]
+    for eager in (True, False):
+        for t in (st.x, st.dW_gu, st.dW_down, st.dx):
+            t.fill_(1.0)
+        out_h.zero_()
+        if eager:
+            dx = st.step(x0_h, up_h, accumulate=False, out=out_h)
+        else:
+            graph = st.capture_step(x0_h, up_h, accumulate=False, out=out_h)
+            out_h.zero_()
+            st.dx.fill_(1.0)
+            graph.replay()
+            dx = st.dx[cfg["L"] % 2]
+        torch.cuda.synchronize()
+        st.ctx.check_status()
+        assert torch.equal(st.x[cfg["L"]], ref[0]) and torch.equal(out_h.cuda(), ref[0])
+        assert torch.equal(st.dW_gu, ref[1]) and torch.equal(st.dW_down, ref[2])
+        assert torch.equal(dx, dx_ref)
+    st.close()
+
+
 def test_empty_batch():
     import torch
     cfg = small_cfg()
