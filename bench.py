@@ -51,7 +51,8 @@ def _peaks():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clocks and throttle reasons with nvidia-smi every 50 ms; the summary covers the
+    samples that arrived between ``begin()`` and ``end()`` (the timed region)."""
 
     FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
               "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
@@ -61,12 +62,19 @@ class ClockSampler:
         self.gpu_index = gpu_index
         self.proc = None
         self.lines = []
+        self.t_begin = self.t_end = None
+
+    def begin(self):
+        self.t_begin = time.perf_counter()
+
+    def end(self):
+        self.t_end = time.perf_counter()
 
     def start(self):
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.gpu_index), f"--query-gpu={self.FIELDS}",
-                 "--format=csv,noheader,nounits", "-lms", "200"],
+                 "--format=csv,noheader,nounits", "-lms", "50"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -75,12 +83,12 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.lines.append(line.strip())
+            self.lines.append((time.perf_counter(), line.strip()))
 
     def stop(self):
         if self.proc is None:
             return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
-        time.sleep(0.25)
+        time.sleep(0.1)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
@@ -88,7 +96,8 @@ class ClockSampler:
             self.proc.kill()
         sm, smax, reasons, power = [], [], set(), []
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for line in self.lines:
+        inside = [l for t, l in self.lines if self.t_begin is not None and self.t_begin <= t <= self.t_end]
+        for line in inside or [l for _, l in self.lines]:
             parts = [p.strip() for p in line.split(",")]
             if len(parts) < 9:
                 continue
@@ -101,7 +110,8 @@ class ClockSampler:
                     reasons.add(name)
         sm.sort()
         return dict(sm_mhz=sm[len(sm) // 2] if sm else None, sm_max_mhz=max(smax) if smax else None,
-                    power_w_max=max(power) if power else None, samples=len(sm), reasons=sorted(reasons))
+                    power_w_max=max(power) if power else None, samples=len(sm),
+                    window="timed region" if inside else "whole run", reasons=sorted(reasons))
 
 
 def algorithmic_bytes(cfg, cap_rows):
@@ -201,6 +211,9 @@ def run_ours(args):
             loss_host.copy_(st.loss, non_blocking=True)
     else:
         eager_step = device_step
+    sampler = ClockSampler(local_rank)               # started ahead of the warm-up: the first sample takes a while
+    if rank == 0 and not args.kernels_only:
+        sampler.start()
     for _ in range(max(args.warmup, 3)):
         device_step()
     st.ctx.check_status()
@@ -211,10 +224,9 @@ def run_ours(args):
         if rank == 0:
             print(json.dumps({"kernels_only": True, "workload": args.workload, "steps": args.steps}))
         return
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
+    sampler.begin()
     ms_total = timed(device_step, args.steps)
+    sampler.end()
     clocks = sampler.stop() if rank == 0 else None
 
     # per-kernel durations, measured live with CUDA events on the launch stream
