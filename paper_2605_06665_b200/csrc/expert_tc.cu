@@ -32,7 +32,9 @@ constexpr uint32_t kBBytes = BN * BK * 2;
 constexpr uint32_t kStageBytes = kABytes + kBBytes;
 constexpr uint32_t kMnBlockBytes = 64 * BK * 2;   // one 64(MN) x 64(K) box
 constexpr uint32_t kBarOffset = 229376;           // operand stages + epilogue staging fill this much
-constexpr uint32_t kSmemTotal = kBarOffset + 512 + 1024;   // + barriers + alignment slack
+constexpr uint32_t kTableBytes = (UNIPOOL_MAX_EXPERTS + 8) * sizeof(uint16_t);   // one 16-bit count per expert
+constexpr uint32_t kSmemTotal = kBarOffset + 512 + kTableBytes + 1024;   // + barriers + table + alignment slack
+static_assert(kSmemTotal <= 227 * 1024, "shared-memory budget");
 constexpr int kChunk = 32;       // output columns one epilogue step moves (a 32 x 32 box per warp)
 constexpr uint32_t kBf16ChunkBytes = 32 * kChunk * 2;      // 2 KiB, 64-byte rows, 64-byte swizzle
 constexpr uint32_t kF32ChunkBytes = 32 * kChunk * 4;       // 4 KiB, 128-byte rows, 128-byte swizzle
@@ -49,6 +51,8 @@ struct GemmParams {
   const int32_t* offsets;       // row tiles: &offsets[n_experts]; wgrad: [n_layers][n_experts+1]
   const int32_t* tile_expert;   // row tiles only
   const int32_t* group_offsets; // row tiles on CTA pairs: [n_experts + 1] starts of the groups
+  int part;                     // row tiles: 0 = every tile; 1 = pair kernel, whole pairs only (a group's odd last
+                                // tile is left out); 2 = single-CTA kernel, only those odd last tiles
   int n_experts, expert_base;
   int n_layers;                 // wgrad
   int layer_stride_rows;        // wgrad
@@ -75,10 +79,13 @@ template <int MODE> struct Traits {
 
 struct TileCoord { int e, mt, nt, kblocks; bool valid; };
 
+// `odd` (row tiles with p.part == 2): odd[e] = groups before expert e that have an odd number of row
+// tiles; the kernel then visits only the last tile of those groups.
 template <int MODE>
-__device__ __forceinline__ int tiles_total(const GemmParams& p, int& n_nt, int& n_mt) {
+__device__ __forceinline__ int tiles_total(const GemmParams& p, int& n_nt, int& n_mt, const uint16_t* odd) {
   if constexpr (Traits<MODE>::kRowTiles) {
     n_mt = p.offsets ? *p.offsets / BM : p.Mdim;     // no offsets: one group of Mdim row tiles
+    if (p.part == 2) n_mt = odd[p.n_experts];
     const int ncols = MODE == kFwd1 ? BN / 2 : BN;
     n_nt = (p.Ndim + ncols - 1) / ncols;
     return n_mt * n_nt;
@@ -90,9 +97,24 @@ __device__ __forceinline__ int tiles_total(const GemmParams& p, int& n_nt, int& 
 }
 
 template <int MODE>
-__device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int tile, int n_nt, int n_mt) {
+__device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int tile, int n_nt, int n_mt,
+                                                const uint16_t* odd = nullptr) {
   TileCoord c;
   if constexpr (Traits<MODE>::kRowTiles) {
+    if (p.part == 2) {                               // the j-th odd group's last tile
+      const int j = tile / n_nt;
+      int lo = 0, hi = p.n_experts - 1;              // last e with odd[e] <= j: the group itself is odd
+      while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if ((int)odd[mid] <= j) lo = mid; else hi = mid - 1;
+      }
+      c.e = lo;
+      c.mt = p.group_offsets[lo + 1] / BM - 1;
+      c.nt = tile % n_nt;
+      c.kblocks = p.Kdim / BK;
+      c.valid = true;
+      return c;
+    }
     // A kernel that consumes what the previous launch produced in ascending row order (the down
     // projection reads A, the second dgrad reads dGU) walks the rows downwards: the rows written
     // last are the ones still in L2.
@@ -311,8 +333,19 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
   tc::tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_ptr;
 
+  uint16_t* odd = reinterpret_cast<uint16_t*>(smem + kBarOffset + 512);     // [n_experts + 1], row tiles with part == 2
+  if constexpr (TR::kRowTiles) {
+    if (p.part == 2) {
+      for (int e = threadIdx.x; e <= p.n_experts; e += blockDim.x) {
+        int before = 0;
+        for (int o = 0; o < e; ++o) before += ((p.group_offsets[o + 1] - p.group_offsets[o]) / BM) & 1;
+        odd[e] = (uint16_t)before;
+      }
+      __syncthreads();
+    }
+  }
   int n_nt, n_mt;
-  const int total = tiles_total<MODE>(p, n_nt, n_mt);
+  const int total = tiles_total<MODE>(p, n_nt, n_mt, odd);
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
@@ -321,7 +354,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
       uint32_t phase = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
-        const TileCoord c = tile_coord<MODE>(p, tile, n_nt, n_mt);
+        const TileCoord c = tile_coord<MODE>(p, tile, n_nt, n_mt, odd);
         if (!c.valid) continue;
         const int pe = p.expert_base + c.e;
         int layer = 0, r = 0, r_end = 0;              // wgrad: walks the rows of expert e, layer by layer
@@ -387,7 +420,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
       int local = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
-        const TileCoord c = tile_coord<MODE>(p, tile, n_nt, n_mt);
+        const TileCoord c = tile_coord<MODE>(p, tile, n_nt, n_mt, odd);
         if (!c.valid) continue;
         const int acc = local & 1;
         const uint32_t acc_phase = (local >> 1) & 1;
@@ -473,7 +506,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     int local = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
-      const TileCoord c = tile_coord<MODE>(p, tile, n_nt, n_mt);
+      const TileCoord c = tile_coord<MODE>(p, tile, n_nt, n_mt, odd);
       if (!c.valid) {
         if constexpr (MODE == kWgrad) {
           if (p.overwrite) {                           // no rows anywhere: the gradient of this tile is zero
@@ -604,8 +637,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
 // even CTA issues the MMAs; every TMA load counts its bytes on the even CTA's mbarrier (plain
 // loads, no multicast); tcgen05.commit arrives on the stage / accumulator barriers of both CTAs.
 constexpr int kPairStages = 6;
-constexpr uint32_t kPairSmemTotal = kSmemTotal + (UNIPOOL_MAX_EXPERTS + 8) * sizeof(uint16_t);   // + one entry per expert
-static_assert(kPairSmemTotal <= 227 * 1024, "shared-memory budget");
+constexpr uint32_t kPairSmemTotal = kSmemTotal;
 constexpr uint32_t kPairHalfBytes = 128 * BK * 2;            // 128 (M or N) x 64 (K) bf16
 constexpr uint32_t kPairStageBytes = 2 * kPairHalfBytes;
 static_assert(kPairStages * kPairStageBytes + kEpiWarps * 8192 == kBarOffset, "shared-memory budget");
@@ -950,7 +982,8 @@ row_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   // pair-tiles before each expert: an expert of n row tiles takes ceil(n / 2)
   for (int e = threadIdx.x; e <= p.n_experts; e += blockDim.x) {
     int before = 0;
-    for (int o = 0; o < e; ++o) before += ((p.group_offsets[o + 1] - p.group_offsets[o]) / BM + 1) >> 1;
+    const int round_up = p.part == 1 ? 0 : 1;        // part 1: a group's odd last tile is another kernel's
+    for (int o = 0; o < e; ++o) before += ((p.group_offsets[o + 1] - p.group_offsets[o]) / BM + round_up) >> 1;
     pp[e] = (uint16_t)before;
   }
   tc::tc_fence_before_sync();
@@ -1085,27 +1118,45 @@ int launch(unipool_ctx* ctx, int phase, const CUtensorMap& tmA, const CUtensorMa
   return UNIPOOL_OK;
 }
 
-// Row-tile GEMMs run on CTA pairs (UNIPOOL_ROW_PAIR=0, a debugging aid, selects the single-CTA
-// kernel); the pair schedule keeps 16-bit counts of pair-tiles.
-// A group of an odd number of row tiles wastes half of its last pair (tensor work and power), so
-// pairs pay once groups are many tiles long: measured neutral to slightly worse at 3 - 7 tiles per
-// group, 10 % faster per GEMM at 32.  They are used when a batch of max_tokens gives the average
-// expert at least eight row tiles (UNIPOOL_ROW_PAIR=1 forces them on, =0 off).
-bool rows_on_pairs(const unipool_ctx* ctx, int n_experts) {
-  static const int forced = [] { const char* v = getenv("UNIPOOL_ROW_PAIR"); return v ? (v[0] == '0' ? 0 : 1) : -1; }();
-  if (ctx->sm_count < 2 || ctx->row_capacity / (2 * BM) + n_experts >= 65535) return false;
-  if (forced >= 0) return forced == 1;
-  return (int64_t)ctx->cfg.max_tokens * ctx->cfg.top_k >= (int64_t)8 * BM * n_experts;
+// How the row-tile GEMMs (gate/up, down, second dgrad) of a call are scheduled:
+//   kRowsSingle  every tile on the single-CTA kernel;
+//   kRowsPairs   every tile on CTA pairs (a group of odd tile count ends in a half-empty pair);
+//   kRowsSplit   whole pairs on the pair kernel, then the odd last tiles on the single-CTA kernel.
+// Pairs move a third fewer operand bytes into the SMs.  Measured (interleaved runs, one B200): 10 %
+// faster per GEMM at 32 row tiles per group, no gain at 3 - 7 tiles, where the half-empty pairs cost
+// what the shared operand saves; the split schedule is 19 % SLOWER than single at 3 tiles per group
+// (the pair kernel's tiles of 12 k-blocks do not reach the single-CTA kernel's rate when most
+// operand bytes miss L2).  So: pairs when a batch of max_tokens gives the average expert eight row
+// tiles, single otherwise; UNIPOOL_ROW_PAIR = 0 / 1 / 2 forces single / pairs / split (a debugging
+// aid).  The pair schedule keeps 16-bit counts of pair-tiles.
+enum RowPlan { kRowsSingle = 0, kRowsPairs = 1, kRowsSplit = 2 };
+RowPlan row_plan(const unipool_ctx* ctx, int n_experts) {
+  static const int forced = [] { const char* v = getenv("UNIPOOL_ROW_PAIR"); return v ? v[0] - '0' : -1; }();
+  if (ctx->sm_count < 2 || ctx->row_capacity / (2 * BM) + n_experts >= 65535) return kRowsSingle;
+  if (forced >= 0 && forced <= 2) return static_cast<RowPlan>(forced);
+  return (int64_t)ctx->cfg.max_tokens * ctx->cfg.top_k >= (int64_t)8 * BM * n_experts ? kRowsPairs : kRowsSingle;
 }
 
+// One row-tile GEMM under `plan`.  tmB: the B map of the single-CTA kernel, tmBp: that of the pair kernel.
 template <int MODE>
-int launch_row_pairs(unipool_ctx* ctx, int phase, const CUtensorMap& tmA, const CUtensorMap& tmB,
-                     const CUtensorMap& tmC0, const CUtensorMap& tmC1, const GemmParams& p, cudaStream_t s) {
-  PhaseTimer pt(ctx, phase, 1, s);
-  auto kern = row_pair_kernel<MODE>;
-  UP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPairSmemTotal));
-  kern<<<ctx->sm_count / 2 * 2, kRowPairThreads, kPairSmemTotal, s>>>(tmA, tmB, tmC0, tmC1, p);
-  UP_LAUNCH_CHECK();
+int launch_rows(unipool_ctx* ctx, int phase, RowPlan plan, const CUtensorMap& tmA, const CUtensorMap& tmB,
+                const CUtensorMap& tmBp, const CUtensorMap& tmC0, const CUtensorMap& tmC1, GemmParams p,
+                cudaStream_t s) {
+  PhaseTimer pt(ctx, phase, plan == kRowsSplit ? 2 : 1, s);
+  if (plan != kRowsSingle) {
+    p.part = plan == kRowsSplit ? 1 : 0;
+    auto kern = row_pair_kernel<MODE>;
+    UP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPairSmemTotal));
+    kern<<<ctx->sm_count / 2 * 2, kRowPairThreads, kPairSmemTotal, s>>>(tmA, tmBp, tmC0, tmC1, p);
+    UP_LAUNCH_CHECK();
+  }
+  if (plan != kRowsPairs) {
+    p.part = plan == kRowsSplit ? 2 : 0;
+    auto kern = grouped_gemm_tc_kernel<MODE>;
+    UP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemTotal));
+    kern<<<ctx->sm_count, Traits<MODE>::kThreads, kSmemTotal, s>>>(tmA, tmB, tmC0, tmC1, p);
+    UP_LAUNCH_CHECK();
+  }
   return UNIPOOL_OK;
 }
 
@@ -1180,16 +1231,15 @@ int expert_fwd_tc(unipool_ctx* ctx, const ExpertFwdArgs& a, cudaStream_t s) {
   p.f = f;
   p.status = ctx->ws.status;
   p.group_offsets = a.offsets;
-  const bool pairs = rows_on_pairs(ctx, a.n_experts);
-  CUtensorMap tmA, tmB, tmC0, tmC1;
+  const RowPlan plan = row_plan(ctx, a.n_experts);
+  CUtensorMap tmA, tmB, tmBp, tmC0, tmC1;
   int rc;
   // GU = Xp [W_gate; W_up]^T with the SwiGLU epilogue.  B tile = 128 gate rows + 128 up rows of the
   // same features, fetched as one 3-D box over W_gu viewed as [2M, f, d] (CTA pairs: one half each,
   // 128 rows of W_gu viewed as [2M f, d]).
   if ((rc = map_2d(ctx, &tmA, a.Xp, d, cap, 64, BM)) != UNIPOOL_OK) return rc;
-  if (pairs) {
-    if ((rc = map_2d(ctx, &tmB, a.W_gu, d, (uint64_t)M * 2 * f, 64, BN / 2)) != UNIPOOL_OK) return rc;
-  } else {
+  if ((rc = map_2d(ctx, &tmBp, a.W_gu, d, (uint64_t)M * 2 * f, 64, BN / 2)) != UNIPOOL_OK) return rc;
+  {
     const uint64_t dims[3] = {(uint64_t)d, (uint64_t)f, (uint64_t)2 * M};
     const uint64_t strides[2] = {(uint64_t)d, (uint64_t)f * d};
     const uint32_t box[3] = {64, BN / 2, 2};
@@ -1198,16 +1248,15 @@ int expert_fwd_tc(unipool_ctx* ctx, const ExpertFwdArgs& a, cudaStream_t s) {
   if ((rc = map_chunk(ctx, &tmC0, a.GU, 2 * f, cap, kMapBf16Chunk)) != UNIPOOL_OK) return rc;
   if ((rc = map_chunk(ctx, &tmC1, a.A, f, cap, kMapBf16Chunk)) != UNIPOOL_OK) return rc;
   p.Ndim = f; p.Kdim = d;
-  rc = pairs ? launch_row_pairs<kFwd1>(ctx, UNIPOOL_PH_EXPERT_FWD_GU, tmA, tmB, tmC0, tmC1, p, s)
-             : launch<kFwd1>(ctx, UNIPOOL_PH_EXPERT_FWD_GU, tmA, tmB, tmC0, tmC1, p, s);
-  if (rc != UNIPOOL_OK) return rc;
+  if ((rc = launch_rows<kFwd1>(ctx, UNIPOOL_PH_EXPERT_FWD_GU, plan, tmA, tmB, tmBp, tmC0, tmC1, p, s)) != UNIPOOL_OK)
+    return rc;
   // Yp = A W_down^T
   if ((rc = map_2d(ctx, &tmA, a.A, f, cap, 64, BM)) != UNIPOOL_OK) return rc;
-  if ((rc = map_2d(ctx, &tmB, a.W_down, f, (uint64_t)M * d, 64, pairs ? BN / 2 : BN)) != UNIPOOL_OK) return rc;
+  if ((rc = map_2d(ctx, &tmB, a.W_down, f, (uint64_t)M * d, 64, BN)) != UNIPOOL_OK) return rc;
+  if ((rc = map_2d(ctx, &tmBp, a.W_down, f, (uint64_t)M * d, 64, BN / 2)) != UNIPOOL_OK) return rc;
   if ((rc = map_chunk(ctx, &tmC0, a.Yp, d, cap, kMapBf16Chunk)) != UNIPOOL_OK) return rc;
   p.Ndim = d; p.Kdim = f;
-  return pairs ? launch_row_pairs<kFwd2>(ctx, UNIPOOL_PH_EXPERT_FWD_DOWN, tmA, tmB, tmC0, tmC0, p, s)
-               : launch<kFwd2>(ctx, UNIPOOL_PH_EXPERT_FWD_DOWN, tmA, tmB, tmC0, tmC0, p, s);
+  return launch_rows<kFwd2>(ctx, UNIPOOL_PH_EXPERT_FWD_DOWN, plan, tmA, tmB, tmBp, tmC0, tmC0, p, s);
 }
 
 int expert_bwd_tc(unipool_ctx* ctx, const ExpertBwdArgs& a, cudaStream_t s) {
@@ -1235,8 +1284,7 @@ int expert_bwd_tc(unipool_ctx* ctx, const ExpertBwdArgs& a, cudaStream_t s) {
   if ((rc = map_chunk(ctx, &tmC0, a.dXp, d, cap, kMapBf16Chunk)) != UNIPOOL_OK) return rc;
   p.Ndim = d; p.Kdim = 2 * f; p.overwrite = 1;
   p.group_offsets = a.offsets;
-  rc = rows_on_pairs(ctx, a.n_experts) ? launch_row_pairs<kDgrad2>(ctx, UNIPOOL_PH_DGRAD_GU, tmA, tmB, tmC0, tmC0, p, s)
-                                       : launch<kDgrad2>(ctx, UNIPOOL_PH_DGRAD_GU, tmA, tmB, tmC0, tmC0, p, s);
+  rc = launch_rows<kDgrad2>(ctx, UNIPOOL_PH_DGRAD_GU, row_plan(ctx, a.n_experts), tmA, tmB, tmB, tmC0, tmC0, p, s);
   if (rc != UNIPOOL_OK) return rc;
   if (a.wgrad) {
     PoolWgradArgs w{1, 0, a.offsets, a.Xp, a.A, a.dYp, a.dGU, a.expert_base, a.n_experts, a.dW_gu, a.dW_down,
