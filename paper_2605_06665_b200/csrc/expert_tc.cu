@@ -651,6 +651,11 @@ __device__ __forceinline__ int wgrad_kblocks(const GemmParams& p, int e) {
   return kb;
 }
 
+// Tile of `pair` in `round` when a sorted tile list is dealt out forwards and backwards alternately.
+__device__ __forceinline__ int snake_tile(int round, int pair, int n_pairs) {
+  return round * n_pairs + ((round & 1) ? n_pairs - 1 - pair : pair);
+}
+
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 wgrad_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                   const __grid_constant__ CUtensorMap tmC0, const GemmParams p) {
@@ -691,8 +696,9 @@ wgrad_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   const int total = p.n_experts * per_e;
 
   // Ragged groups: the contraction length of a tile is its expert's row count over all layers.  The
-  // experts are taken in order of decreasing length (ties by index), so that the round-robin over the
-  // CTA pairs deals out tiles of similar size in every round and the long ones first.
+  // experts are taken in order of decreasing length (ties by index) and dealt to the CTA pairs
+  // boustrophedon-wise (round 0: pair 0 .. P-1, round 1: pair P-1 .. 0, ...), so that every round holds
+  // tiles of similar size, the long ones come first, and no pair collects the longest tile of every round.
   uint16_t* order = reinterpret_cast<uint16_t*>(smem + kBarOffset + 512);   // [n_experts] i-th longest expert
   int* kb_of = reinterpret_cast<int*>(smem + kPairStages * kPairStageBytes);  // scratch in the (still idle) staging tiles
   for (int e = threadIdx.x; e < p.n_experts; e += blockDim.x) kb_of[e] = wgrad_kblocks(p, e);
@@ -714,7 +720,9 @@ wgrad_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int tile = pair; tile < total && ok; tile += n_pairs) {
+      for (int round = 0; round * n_pairs < total && ok; ++round) {
+        const int tile = snake_tile(round, pair, n_pairs);
+        if (tile >= total) continue;
         const int e = order[tile / per_e], rem = tile % per_e, mt = rem / n_nt, nt = rem % n_nt;
         const int kblocks = wgrad_kblocks(p, e);
         int layer = 0, r = p.offsets[e], r_end = p.offsets[e + 1];
@@ -751,7 +759,9 @@ wgrad_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       uint32_t phase = 0;
       int local = 0;
       bool ok = true;
-      for (int tile = pair; tile < total && ok; tile += n_pairs) {
+      for (int round = 0; round * n_pairs < total && ok; ++round) {
+        const int tile = snake_tile(round, pair, n_pairs);
+        if (tile >= total) continue;
         const int kblocks = wgrad_kblocks(p, order[tile / per_e]);
         if (kblocks == 0) continue;
         const int acc = local & 1;
@@ -780,7 +790,9 @@ wgrad_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     const int quarter = warp & 3;
     uint8_t* stg = smem + kPairStages * kPairStageBytes + (warp - 2) * 8192;
     int gchunk = 0, local = 0;
-    for (int tile = pair; tile < total; tile += n_pairs) {
+    for (int round = 0; round * n_pairs < total; ++round) {
+      const int tile = snake_tile(round, pair, n_pairs);
+      if (tile >= total) continue;
       const int e = order[tile / per_e], rem = tile % per_e, mt = rem / n_nt, nt = rem % n_nt;
       const int m0 = mt * 256 + rank * 128 + quarter * 32;
       const int grow = (p.expert_base + e) * p.Mdim + m0;
