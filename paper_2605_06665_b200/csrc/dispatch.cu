@@ -237,7 +237,9 @@ combine_kernel(const uint4* __restrict__ Yp, const int32_t* __restrict__ row_of,
 
 // Backward of the combine, token-major: for token t and slot j with row r = row_of[t,j]
 //   dgate[t,j] = <dy[t], Yp[r]>,   dYp[r] = gate[t,j] * dy[t];
-// afterwards the pad rows (token_of < 0) below offsets[M] are zeroed.
+// afterwards the pad rows (token_of < 0) below offsets[M] are zeroed.  A warp takes KT slots of one
+// token; with k > KT the token's slots are split over ceil(k / KT) warps (each re-reads dy[t], which
+// keeps the registers per thread low enough for four resident blocks per SM).
 template <typename T, int KT>
 __global__ void __launch_bounds__(256)
 combine_bwd_kernel(const uint4* __restrict__ dy, const uint4* __restrict__ Yp,
@@ -246,13 +248,15 @@ combine_bwd_kernel(const uint4* __restrict__ dy, const uint4* __restrict__ Yp,
                    uint4* __restrict__ dYp, float* __restrict__ dgate, int n_tokens, int k, int row_vecs) {
   constexpr int N = Vec16<T>::N;
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-  for (int t = blockIdx.x * 8 + warp; t < n_tokens; t += gridDim.x * 8) {
+  const int groups = (k + KT - 1) / KT;
+  for (int64_t item = blockIdx.x * 8 + warp; item < (int64_t)n_tokens * groups; item += gridDim.x * 8) {
+    const int t = (int)(item / groups), j0 = (int)(item % groups) * KT;
     int rows[KT];
     float g[KT], dot[KT];
 #pragma unroll
     for (int j = 0; j < KT; ++j) {
-      rows[j] = j < k ? row_of[(int64_t)t * k + j] : -1;
-      g[j] = j < k ? gate[(int64_t)t * k + j] : 0.f;
+      rows[j] = j0 + j < k ? row_of[(int64_t)t * k + j0 + j] : -1;
+      g[j] = j0 + j < k ? gate[(int64_t)t * k + j0 + j] : 0.f;
       dot[j] = 0.f;
     }
     for (int v0 = lane; v0 < row_vecs; v0 += 32 * kVpl) {
@@ -290,7 +294,7 @@ combine_bwd_kernel(const uint4* __restrict__ dy, const uint4* __restrict__ Yp,
     for (int j = 0; j < KT; ++j) {
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) dot[j] += __shfl_xor_sync(0xffffffffu, dot[j], o);
-      if (lane == 0 && j < k) dgate[(int64_t)t * k + j] = dot[j];
+      if (lane == 0 && j0 + j < k) dgate[(int64_t)t * k + j0 + j] = dot[j];
     }
   }
   const int used = *offsets_end;
@@ -384,9 +388,7 @@ static void combine_bwd_dispatch_k(int grid, cudaStream_t s, int k, const void* 
   auto Y = static_cast<const uint4*>(Yp);
   auto O = static_cast<uint4*>(dYp);
   if (k <= 1) combine_bwd_kernel<T, 1><<<grid, 256, 0, s>>>(D, Y, row_of, gate, token_of, offsets_end, O, dgate, n_tokens, k, row_vecs);
-  else if (k <= 2) combine_bwd_kernel<T, 2><<<grid, 256, 0, s>>>(D, Y, row_of, gate, token_of, offsets_end, O, dgate, n_tokens, k, row_vecs);
-  else if (k <= 4) combine_bwd_kernel<T, 4><<<grid, 256, 0, s>>>(D, Y, row_of, gate, token_of, offsets_end, O, dgate, n_tokens, k, row_vecs);
-  else combine_bwd_kernel<T, 8><<<grid, 256, 0, s>>>(D, Y, row_of, gate, token_of, offsets_end, O, dgate, n_tokens, k, row_vecs);
+  else combine_bwd_kernel<T, 2><<<grid, 256, 0, s>>>(D, Y, row_of, gate, token_of, offsets_end, O, dgate, n_tokens, k, row_vecs);
 }
 
 int combine_bwd_launch(unipool_ctx* ctx, const void* dy, int T, const int32_t* row_of,
@@ -395,7 +397,7 @@ int combine_bwd_launch(unipool_ctx* ctx, const void* dy, int T, const int32_t* r
   if (T == 0) return UNIPOOL_OK;
   const int k = ctx->cfg.top_k;
   const int row_vecs = (int)((size_t)ctx->cfg.d_model * ctx->elem_bytes / 16);
-  const int grid = row_mover_grid(ctx, T);
+  const int grid = row_mover_grid(ctx, (int64_t)T * ((k + 1) / 2));     // one warp per token and pair of slots
   PhaseTimer pt(ctx, UNIPOOL_PH_BWD_SCALE_GATHER, 1, s);
   if (ctx->cfg.dtype == UNIPOOL_BF16)
     combine_bwd_dispatch_k<__nv_bfloat16>(grid, s, k, dy, Yp, row_of, gate, token_of, offsets + M, dYp, dgate, T, row_vecs);
