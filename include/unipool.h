@@ -154,7 +154,7 @@ int unipool_dispatch(unipool_ctx* ctx, const void* x, int32_t T, const int32_t* 
  * Same inputs, outputs and results as unipool_dispatch, for d_model/dtype/top_k given here and
  * row_capacity = rows of the permuted buffers (a multiple of UNIPOOL_ROW_ALIGN, at least
  * T*top_k + n_experts*(UNIPOOL_ROW_ALIGN-1) rounded up).
- *   - Limit: ceil(T/64) * n_experts <= 524224 (e.g. 65536 tokens at 511 experts); beyond it the
+ *   - Limit: ceil(T/256) * n_experts <= 524224 (e.g. 261888 tokens at 512 experts); beyond it the
  *     call fails with UNIPOOL_ERR_WORKSPACE and launches nothing.
  *   - The first call on each device looks up the array's device address (with that device
  *     current); make that first call outside any stream capture.

@@ -62,7 +62,7 @@ struct Workspace {
   size_t   bytes;         // total
 };
 
-constexpr int kDispatchChunkTokens = 64;   // tokens per dispatch block
+constexpr int kDispatchChunkTokens = 256;  // tokens per dispatch block (eight warps of 32 tokens)
 
 Workspace carve_workspace(const unipool_config& cfg, void* base);
 

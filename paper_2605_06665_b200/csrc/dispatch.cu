@@ -5,27 +5,44 @@
 namespace unipool {
 
 // ---------------------------------------------------------------- maps
-// Block b owns tokens [b*CH, (b+1)*CH); one warp per block so that the stable
-// (token-major) order inside the chunk is the lane order.
-__global__ void __launch_bounds__(32)
+// Block b owns tokens [b*CH, (b+1)*CH), warp w of it the tokens [w*CH/8, (w+1)*CH/8) of those: the
+// stable (token-major) order is block order, then warp order, then lane order inside a warp.
+constexpr int kDispatchWarps = 8;
+constexpr int kDispatchWarpTokens = kDispatchChunkTokens / kDispatchWarps;
+
+// hist[w][e] = assignments to expert e among warp w's tokens (shared memory, [kDispatchWarps][M]).
+// `status` (may be NULL) receives a corrupt routing entry; the assignment is dropped either way.
+__device__ __forceinline__ void chunk_histograms(const int32_t* __restrict__ idx, int T, int k, int M, int* hist,
+                                                 int32_t* status, int64_t& a_begin, int64_t& a_end) {
+  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+  for (int i = threadIdx.x; i < kDispatchWarps * M; i += blockDim.x) hist[i] = 0;
+  __syncthreads();
+  const int64_t total = (int64_t)T * k;
+  a_begin = min(total, ((int64_t)blockIdx.x * kDispatchChunkTokens + (int64_t)warp * kDispatchWarpTokens) * k);
+  a_end = min(total, a_begin + (int64_t)kDispatchWarpTokens * k);
+  for (int64_t a = a_begin + lane; a < a_end; a += 32) {
+    const int e = idx[a];
+    if (e < 0 || e >= M) {          // corrupt routing table: record it, drop the assignment
+      if (status != nullptr && atomicCAS(status, 0, kStatusCheck) == 0) { status[1] = 10; status[2] = e; }
+      continue;
+    }
+    atomicAdd(&hist[warp * M + e], 1);
+  }
+  __syncthreads();
+}
+
+__global__ void __launch_bounds__(kDispatchWarps * 32)
 dispatch_hist_kernel(const int32_t* __restrict__ idx, int T, int k, int M, int32_t* __restrict__ block_hist,
                      int32_t* __restrict__ status) {
   extern __shared__ int hist[];
-  const int lane = threadIdx.x;
-  for (int i = lane; i < M; i += 32) hist[i] = 0;
-  __syncwarp();
-  const int64_t a_begin = (int64_t)blockIdx.x * kDispatchChunkTokens * k;
-  const int64_t a_end = min((int64_t)T * k, a_begin + (int64_t)kDispatchChunkTokens * k);
-  for (int64_t a = a_begin + lane; a < a_end; a += 32) {
-    int e = idx[a];
-    if (e < 0 || e >= M) {          // corrupt routing table: record it, drop the assignment
-      if (atomicCAS(status, 0, kStatusCheck) == 0) { status[1] = 10; status[2] = e; }
-      continue;
-    }
-    atomicAdd(&hist[e], 1);
+  int64_t a_begin, a_end;
+  chunk_histograms(idx, T, k, M, hist, status, a_begin, a_end);
+  for (int e = threadIdx.x; e < M; e += blockDim.x) {
+    int total = 0;
+#pragma unroll
+    for (int w = 0; w < kDispatchWarps; ++w) total += hist[w * M + e];
+    block_hist[(int64_t)blockIdx.x * M + e] = total;
   }
-  __syncwarp();
-  for (int i = lane; i < M; i += 32) block_hist[(int64_t)blockIdx.x * M + i] = hist[i];
 }
 
 // One block of 1024 threads: per-expert totals -> padded exclusive scan -> per-(chunk, expert) bases.
@@ -90,16 +107,28 @@ dispatch_scan_kernel(int32_t* __restrict__ block_hist, int n_blocks, int M, int 
     tile_expert[tl] = -1;
 }
 
-__global__ void __launch_bounds__(32)
+// block_base[b][e] = first row of block b's assignments to expert e (written by the scan).  The
+// block rebuilds its warps' histograms, turns them into each warp's first row per expert, and every
+// warp ranks its assignments in lane order.
+__global__ void __launch_bounds__(kDispatchWarps * 32)
 dispatch_rank_kernel(const int32_t* __restrict__ idx, int T, int k, int M,
                      const int32_t* __restrict__ block_base, int32_t* __restrict__ row_of,
                      int32_t* __restrict__ token_of) {
-  extern __shared__ int next_row[];
-  const int lane = threadIdx.x;
-  for (int i = lane; i < M; i += 32) next_row[i] = block_base[(int64_t)blockIdx.x * M + i];
-  __syncwarp();
-  const int64_t a_begin = (int64_t)blockIdx.x * kDispatchChunkTokens * k;
-  const int64_t a_end = min((int64_t)T * k, a_begin + (int64_t)kDispatchChunkTokens * k);
+  extern __shared__ int hist[];
+  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+  int64_t a_begin, a_end;
+  chunk_histograms(idx, T, k, M, hist, nullptr, a_begin, a_end);
+  for (int e = threadIdx.x; e < M; e += blockDim.x) {
+    int run = block_base[(int64_t)blockIdx.x * M + e];
+#pragma unroll
+    for (int w = 0; w < kDispatchWarps; ++w) {
+      const int n = hist[w * M + e];
+      hist[w * M + e] = run;
+      run += n;
+    }
+  }
+  __syncthreads();
+  int* next_row = hist + warp * M;
   for (int64_t a0 = a_begin; a0 < a_end; a0 += 32) {
     const int64_t a = a0 + lane;
     const bool live = a < a_end;
@@ -249,8 +278,9 @@ combine_bwd_kernel(const uint4* __restrict__ dy, const uint4* __restrict__ Yp,
   constexpr int N = Vec16<T>::N;
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
   const int groups = (k + KT - 1) / KT;
-  for (int64_t item = blockIdx.x * 8 + warp; item < (int64_t)n_tokens * groups; item += gridDim.x * 8) {
-    const int t = (int)(item / groups), j0 = (int)(item % groups) * KT;
+  const int n_items = n_tokens * groups;                 // < 2^30: T * k is
+  for (int item = blockIdx.x * 8 + warp; item < n_items; item += gridDim.x * 8) {
+    const int t = groups == 1 ? item : item / groups, j0 = groups == 1 ? 0 : (item % groups) * KT;
     int rows[KT];
     float g[KT], dot[KT];
 #pragma unroll
@@ -333,11 +363,11 @@ int dispatch_launch(unipool_ctx* ctx, const void* x, int T, const int32_t* idx, 
   int32_t* bh = ctx->ws.block_hist;
   {
   PhaseTimer pt(ctx, UNIPOOL_PH_DISPATCH_MAPS, 3, s);
-  dispatch_hist_kernel<<<n_blocks, 32, M * sizeof(int), s>>>(idx, T, k, M, bh, ctx->ws.status);
+  dispatch_hist_kernel<<<n_blocks, kDispatchWarps * 32, kDispatchWarps * M * sizeof(int), s>>>(idx, T, k, M, bh, ctx->ws.status);
   UP_LAUNCH_CHECK();
   dispatch_scan_kernel<<<1, kScanThreads, 0, s>>>(bh, n_blocks, M, cap, offsets, token_of, tile_expert);
   UP_LAUNCH_CHECK();
-  dispatch_rank_kernel<<<n_blocks, 32, M * sizeof(int), s>>>(idx, T, k, M, bh, row_of, token_of);
+  dispatch_rank_kernel<<<n_blocks, kDispatchWarps * 32, kDispatchWarps * M * sizeof(int), s>>>(idx, T, k, M, bh, row_of, token_of);
   UP_LAUNCH_CHECK();
   }
   PhaseTimer pt(ctx, UNIPOOL_PH_DISPATCH_GATHER, 1, s);
@@ -476,11 +506,11 @@ extern "C" int unipool_dispatch_static(const void* x, int32_t T, int32_t d_model
   }
   // the histograms are fully rewritten by the first kernel for the chunks of this call; nothing
   // else in the array has to start at zero
-  dispatch_hist_kernel<<<n_blocks, 32, n_experts * sizeof(int), s>>>(idx, T, top_k, n_experts, bh, status);
+  dispatch_hist_kernel<<<n_blocks, kDispatchWarps * 32, kDispatchWarps * n_experts * sizeof(int), s>>>(idx, T, top_k, n_experts, bh, status);
   UP_LAUNCH_CHECK();
   dispatch_scan_kernel<<<1, kScanThreads, 0, s>>>(bh, n_blocks, n_experts, cap, offsets, token_of, tile_expert);
   UP_LAUNCH_CHECK();
-  dispatch_rank_kernel<<<n_blocks, 32, n_experts * sizeof(int), s>>>(idx, T, top_k, n_experts, bh, row_of, token_of);
+  dispatch_rank_kernel<<<n_blocks, kDispatchWarps * 32, kDispatchWarps * n_experts * sizeof(int), s>>>(idx, T, top_k, n_experts, bh, row_of, token_of);
   UP_LAUNCH_CHECK();
   const int row_vecs = (int)((size_t)d_model * eb / 16);
   int64_t want = ((int64_t)cap + 7) / 8, lim = (int64_t)g_scratch_sms[dev] * 8;

@@ -62,7 +62,7 @@ def test_dispatch_static_refuses_what_does_not_fit():
     import torch
     from paper_2605_06665_b200 import binding as B
     d, k, M = 64, 1, 512
-    T = 70000                                    # ceil(T/64) * 512 entries > the built-in scratch
+    T = 270000                                   # ceil(T/256) * 512 entries > the built-in scratch
     cap = (T * k + M * 127 + 127) // 128 * 128
     one = torch.zeros(16, dtype=torch.int32, device="cuda")
     with pytest.raises(B.UniPoolError) as ei:
