@@ -270,7 +270,7 @@ combine_kernel(const uint4* __restrict__ Yp, const int32_t* __restrict__ row_of,
 // token; with k > KT the token's slots are split over ceil(k / KT) warps (each re-reads dy[t], which
 // keeps the registers per thread low enough for four resident blocks per SM).
 template <typename T, int KT>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 4)
 combine_bwd_kernel(const uint4* __restrict__ dy, const uint4* __restrict__ Yp,
                    const int32_t* __restrict__ row_of, const float* __restrict__ gate,
                    const int32_t* __restrict__ token_of, const int32_t* __restrict__ offsets_end,
