@@ -314,16 +314,34 @@ route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       __threadfence();
       double* dsum = reinterpret_cast<double*>(zstage);  // [4][M] in the z staging tiles (they have drained)
       int* csum = reinterpret_cast<int*>(zstage + 4 * UNIPOOL_MAX_EXPERTS * sizeof(double));   // [4][M]
-      for (int i = lane; i < M; i += 32) {
-        int cnt = 0;
-        double sum = 0.0;
+      if ((M & 3) == 0) {                  // 16-byte rows: a lane takes four neighbouring experts per load
+        for (int i = 4 * lane; i < M; i += 128) {
+          int4 cnt = make_int4(0, 0, 0, 0);
+          double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
 #pragma unroll 8
-        for (int b = warp; b < (int)gridDim.x; b += 4) {
-          cnt += __ldcg(&p.part_counts[(int64_t)b * M + i]);
-          sum += (double)__ldcg(&p.part_sums[(int64_t)b * M + i]);
+          for (int b = warp; b < (int)gridDim.x; b += 4) {
+            const int4 c = __ldcg(reinterpret_cast<const int4*>(p.part_counts + (int64_t)b * M + i));
+            const float4 v = __ldcg(reinterpret_cast<const float4*>(p.part_sums + (int64_t)b * M + i));
+            cnt.x += c.x; cnt.y += c.y; cnt.z += c.z; cnt.w += c.w;
+            s0 += (double)v.x; s1 += (double)v.y; s2 += (double)v.z; s3 += (double)v.w;
+          }
+          csum[warp * M + i] = cnt.x; csum[warp * M + i + 1] = cnt.y;
+          csum[warp * M + i + 2] = cnt.z; csum[warp * M + i + 3] = cnt.w;
+          dsum[warp * M + i] = s0; dsum[warp * M + i + 1] = s1;
+          dsum[warp * M + i + 2] = s2; dsum[warp * M + i + 3] = s3;
         }
-        csum[warp * M + i] = cnt;
-        dsum[warp * M + i] = sum;
+      } else {
+        for (int i = lane; i < M; i += 32) {
+          int cnt = 0;
+          double sum = 0.0;
+#pragma unroll 8
+          for (int b = warp; b < (int)gridDim.x; b += 4) {
+            cnt += __ldcg(&p.part_counts[(int64_t)b * M + i]);
+            sum += (double)__ldcg(&p.part_sums[(int64_t)b * M + i]);
+          }
+          csum[warp * M + i] = cnt;
+          dsum[warp * M + i] = sum;
+        }
       }
       asm volatile("bar.sync 1, 128;" ::: "memory");
       for (int i = threadIdx.x; i < M; i += kTile) {

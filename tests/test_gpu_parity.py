@@ -190,6 +190,22 @@ def test_softmax_router_mode(kw, T):
     run_layer_checks(cfg, T, cfg["L"], seed=6)
 
 
+@pytest.mark.parametrize("plan", ["1", "2"])
+def test_forced_row_gemm_schedules(plan):
+    """The row-tile GEMMs' other schedules (UNIPOOL_ROW_PAIR=1: every tile on CTA pairs, =2: whole
+    pairs on the pair kernel and the odd last tiles on the single-CTA kernel) pass the same bf16
+    parity cases; the switch is read once per process, so the cases run in a child process."""
+    import os
+    import subprocess
+    import sys
+    env = dict(os.environ, UNIPOOL_ROW_PAIR=plan)
+    here = os.path.dirname(os.path.abspath(__file__))
+    r = subprocess.run([sys.executable, "-m", "pytest", os.path.join(here, "test_gpu_parity.py"), "-m", "gpu", "-x", "-q",
+                        "-k", "small_bf16_shapes or softmax_router_mode or deferred_pool_wgrad"],
+                       env=env, cwd=os.path.dirname(here), capture_output=True, text=True, timeout=900)
+    assert r.returncode == 0, r.stdout[-3000:] + r.stderr[-2000:]
+
+
 def test_tiny_fp32_end_to_end():
     """Config 1 without teacher forcing: forward, balance loss and backward of the
     whole 4-layer stack against the float64 oracle."""
