@@ -77,7 +77,7 @@ template <int MODE> struct Traits {
   static constexpr bool kRowTiles = MODE != kWgrad;
 };
 
-struct TileCoord { int e, mt, nt, kblocks; bool valid; };
+struct TileCoord { int e, mt, nt, kblocks; bool valid; int col0, ncols; };   // output columns [col0, col0 + ncols)
 
 // `odd` (row tiles with p.part == 2): odd[e] = groups before expert e that have an odd number of row
 // tiles; the kernel then visits only the last tile of those groups.
@@ -113,6 +113,8 @@ __device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int tile, i
       c.nt = tile % n_nt;
       c.kblocks = p.Kdim / BK;
       c.valid = true;
+      c.col0 = c.nt * BN;
+      c.ncols = BN;
       return c;
     }
     // A kernel that consumes what the previous launch produced in ascending row order (the down
@@ -124,6 +126,8 @@ __device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int tile, i
     c.e = p.tile_expert ? p.tile_expert[c.mt] : 0;
     c.kblocks = p.Kdim / BK;
     c.valid = c.e >= 0 && c.e < p.n_experts;
+    c.col0 = c.nt * BN;
+    c.ncols = BN;
   } else {
     const int per_e = n_mt * n_nt;
     c.e = tile / per_e;
@@ -142,7 +146,39 @@ __device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int tile, i
     }
     c.kblocks = kb;
     c.valid = kb > 0;
+    c.col0 = c.nt * BN;
+    c.ncols = BN;
   }
+  return c;
+}
+
+// The tiles of a launch are dealt round-robin to the CTAs; the last, partial round would keep a few
+// CTAs busy for a whole tile while the rest wait.  For the plain row-tile GEMMs (down projection,
+// second dgrad) the tiles of that round are cut into 2 or 4 column slices (MMA N = 128 or 64) so that
+// they spread over (nearly) all CTAs.  Work units: [0, full) whole tiles, then slices.
+struct TailSplit { int full, slices, units; };
+template <int MODE>
+__device__ __forceinline__ TailSplit tail_split(const GemmParams& p, int total) {
+  TailSplit t{total, 1, total};
+  if constexpr (MODE == kFwd2 || MODE == kDgrad2) {
+    const int grid = (int)gridDim.x;
+    const int rest = total % grid;
+    if (p.part == 0 && rest > 0 && 2 * rest <= grid) {
+      t.full = total - rest;
+      t.slices = 4 * rest <= grid ? 4 : 2;
+      t.units = t.full + rest * t.slices;
+    }
+  }
+  return t;
+}
+template <int MODE>
+__device__ __forceinline__ TileCoord unit_coord(const GemmParams& p, const TailSplit& ts, int unit, int n_nt, int n_mt,
+                                                const uint16_t* odd) {
+  if (unit < ts.full) return tile_coord<MODE>(p, unit, n_nt, n_mt, odd);
+  const int u = unit - ts.full;
+  TileCoord c = tile_coord<MODE>(p, ts.full + u / ts.slices, n_nt, n_mt, odd);
+  c.ncols = BN / ts.slices;
+  c.col0 += (u % ts.slices) * c.ncols;
   return c;
 }
 
@@ -265,11 +301,12 @@ __device__ __forceinline__ void epilogue_swiglu(const CUtensorMap* tmC0, const C
 // Epilogue of a plain row-tile GEMM (down projection, second dgrad) for one warp's 32 rows: the
 // accumulator is rounded to bf16, staged in a ring of four chunk tiles and stored (or add-reduced).
 template <int MODE>
-__device__ __forceinline__ void epilogue_rows(const CUtensorMap* tmC0, const GemmParams& p, uint32_t t_row, int nt,
-                                              int row0, uint8_t* stg, int lane, int& gchunk, int ch0 = 0, int step = 1) {
+__device__ __forceinline__ void epilogue_rows(const CUtensorMap* tmC0, const GemmParams& p, uint32_t t_row, int col0,
+                                              int ncols, int row0, uint8_t* stg, int lane, int& gchunk, int ch0 = 0,
+                                              int step = 1) {
 #pragma unroll 1
-  for (int ch = ch0; ch < BN / kChunk; ch += step) {
-    const int col = nt * BN + ch * kChunk;
+  for (int ch = ch0; ch < ncols / kChunk; ch += step) {
+    const int col = col0 + ch * kChunk;
     if (col >= p.Ndim) break;
     uint32_t rr[32];
     tc::tmem_ld_32x32(t_row + ch * kChunk, rr);
@@ -322,7 +359,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     tc::tma_prefetch_desc(&tmA);
     tc::tma_prefetch_desc(&tmB);
     tc::tma_prefetch_desc(&tmC0);
-    if constexpr (MODE == kFwd1 || MODE == kDgrad1) tc::tma_prefetch_desc(&tmC1);
+    if constexpr (MODE == kFwd1 || MODE == kDgrad1 || MODE == kFwd2) tc::tma_prefetch_desc(&tmC1);
   }
   if (warp == 1) {
     tc::tmem_alloc(tmem_ptr, kTmemCols);
@@ -345,7 +382,9 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     }
   }
   int n_nt, n_mt;
-  const int total = tiles_total<MODE>(p, n_nt, n_mt, odd);
+  const int n_tiles = tiles_total<MODE>(p, n_nt, n_mt, odd);
+  const TailSplit ts = tail_split<MODE>(p, n_tiles);
+  const int total = ts.units;                        // work units: whole tiles, then slices of the last round
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
@@ -354,7 +393,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
       uint32_t phase = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
-        const TileCoord c = tile_coord<MODE>(p, tile, n_nt, n_mt, odd);
+        const TileCoord c = unit_coord<MODE>(p, ts, tile, n_nt, n_mt, odd);
         if (!c.valid) continue;
         const int pe = p.expert_base + c.e;
         int layer = 0, r = 0, r_end = 0;              // wgrad: walks the rows of expert e, layer by layer
@@ -371,19 +410,25 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
           if (!tc::mbar_wait(&empty_bar[stage], phase ^ 1u, abort)) { report_timeout(p, abort, 1); ok = false; break; }
           uint8_t* sA = smem + stage * kStageBytes;
           uint8_t* sB = sA + kABytes;
-          tc::mbar_expect_tx(&full_bar[stage], kStageBytes);
+          tc::mbar_expect_tx(&full_bar[stage], kABytes + (uint32_t)c.ncols * (BK * 2));
           if constexpr (MODE == kFwd1) {
             tc::tma_load_2d(sA, &tmA, &full_bar[stage], kb * BK, c.mt * BM);
             tc::tma_load_3d(sB, &tmB, &full_bar[stage], kb * BK, c.nt * (BN / 2), 2 * pe);
           } else if constexpr (MODE == kFwd2) {
             tc::tma_load_2d(sA, &tmA, &full_bar[stage], kb * BK, c.mt * BM);
-            tc::tma_load_2d(sB, &tmB, &full_bar[stage], kb * BK, pe * p.Ndim + c.nt * BN);
+            if (c.ncols == BN) {
+              tc::tma_load_2d(sB, &tmB, &full_bar[stage], kb * BK, pe * p.Ndim + c.col0);
+            } else {                                  // a column slice: 64-row boxes of the weight (tmC1)
+              for (int i = 0; i < c.ncols / 64; ++i)
+                tc::tma_load_2d(sB + i * kMnBlockBytes, &tmC1, &full_bar[stage], kb * BK, pe * p.Ndim + c.col0 + 64 * i);
+            }
           } else if constexpr (MODE == kDgrad1 || MODE == kDgrad2) {
             tc::tma_load_2d(sA, &tmA, &full_bar[stage], kb * BK, c.mt * BM);
 #pragma unroll
             for (int i = 0; i < BN / 64; ++i)
-              tc::tma_load_2d(sB + i * kMnBlockBytes, &tmB, &full_bar[stage], c.nt * BN + 64 * i,
-                              pe * p.Kdim + kb * BK);
+              if (64 * i < c.ncols)
+                tc::tma_load_2d(sB + i * kMnBlockBytes, &tmB, &full_bar[stage], c.col0 + 64 * i,
+                                pe * p.Kdim + kb * BK);
           } else {
             while (r >= r_end) {                        // next layer that has rows for this expert
               ++layer;
@@ -411,7 +456,6 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc = tc::instr_desc_bf16(BN, TR::kAMn, TR::kBMn);
       constexpr uint32_t a_lbo = TR::kAMn ? kMnBlockBytes : 16, b_lbo = TR::kBMn ? kMnBlockBytes : 16;
       constexpr uint32_t a_step = (TR::kAMn ? 16 * 128 : 32) >> 4;   // descriptor units of 16 bytes per K = 16
       constexpr uint32_t b_step = (TR::kBMn ? 16 * 128 : 32) >> 4;
@@ -420,7 +464,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
       int local = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
-        const TileCoord c = tile_coord<MODE>(p, tile, n_nt, n_mt, odd);
+        const TileCoord c = unit_coord<MODE>(p, ts, tile, n_nt, n_mt, odd);
         if (!c.valid) continue;
         const int acc = local & 1;
         const uint32_t acc_phase = (local >> 1) & 1;
@@ -428,6 +472,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
         if (!tc::mbar_wait(&tmem_empty[acc], acc_phase ^ 1u, abort)) { report_timeout(p, abort, 2); break; }
         tc::tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + acc * BN;
+        const uint32_t idesc = tc::instr_desc_bf16(c.ncols, TR::kAMn, TR::kBMn);
         for (int kb = 0; kb < c.kblocks; ++kb) {
           if (!tc::mbar_wait(&full_bar[stage], phase, abort)) { report_timeout(p, abort, 3); ok = false; break; }
           tc::tc_fence_after_sync();
@@ -506,7 +551,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     int local = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
-      const TileCoord c = tile_coord<MODE>(p, tile, n_nt, n_mt, odd);
+      const TileCoord c = unit_coord<MODE>(p, ts, tile, n_nt, n_mt, odd);
       if (!c.valid) {
         if constexpr (MODE == kWgrad) {
           if (p.overwrite) {                           // no rows anywhere: the gradient of this tile is zero
@@ -549,7 +594,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
       if constexpr (MODE == kFwd1) {
         epilogue_swiglu(&tmC0, &tmC1, p, t_row, c.nt, row0, stg, lane);
       } else if constexpr (MODE == kFwd2 || MODE == kDgrad2) {
-        epilogue_rows<MODE>(&tmC0, p, t_row, c.nt, row0, stg, lane, gchunk);
+        epilogue_rows<MODE>(&tmC0, p, t_row, c.col0, c.ncols, row0, stg, lane, gchunk);
       } else if constexpr (MODE == kDgrad1) {
 #pragma unroll 1
         for (int ch = 0; ch < nch; ++ch) {
@@ -1097,7 +1142,7 @@ row_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         const int row0 = t.mt * BM + quarter * 32;
         constexpr int kShare = kRowPairEpiWarps / 4;     // warps per TMEM lane quarter
         if constexpr (MODE == kFwd1) epilogue_swiglu(&tmC0, &tmC1, p, t_row, t.nt, row0, stg, lane, half, kShare);
-        else epilogue_rows<MODE>(&tmC0, p, t_row, t.nt, row0, stg, lane, gchunk, half, kShare);
+        else epilogue_rows<MODE>(&tmC0, p, t_row, t.nt * BN, BN, row0, stg, lane, gchunk, half, kShare);
       }
       tc::tc_fence_before_sync();
       __syncwarp();
@@ -1266,9 +1311,10 @@ int expert_fwd_tc(unipool_ctx* ctx, const ExpertFwdArgs& a, cudaStream_t s) {
   if ((rc = map_2d(ctx, &tmA, a.A, f, cap, 64, BM)) != UNIPOOL_OK) return rc;
   if ((rc = map_2d(ctx, &tmB, a.W_down, f, (uint64_t)M * d, 64, BN)) != UNIPOOL_OK) return rc;
   if ((rc = map_2d(ctx, &tmBp, a.W_down, f, (uint64_t)M * d, 64, BN / 2)) != UNIPOOL_OK) return rc;
+  if ((rc = map_2d(ctx, &tmC1, a.W_down, f, (uint64_t)M * d, 64, 64)) != UNIPOOL_OK) return rc;   // column slices
   if ((rc = map_chunk(ctx, &tmC0, a.Yp, d, cap, kMapBf16Chunk)) != UNIPOOL_OK) return rc;
   p.Ndim = d; p.Kdim = f;
-  return launch_rows<kFwd2>(ctx, UNIPOOL_PH_EXPERT_FWD_DOWN, plan, tmA, tmB, tmBp, tmC0, tmC0, p, s);
+  return launch_rows<kFwd2>(ctx, UNIPOOL_PH_EXPERT_FWD_DOWN, plan, tmA, tmB, tmBp, tmC0, tmC1, p, s);
 }
 
 int expert_bwd_tc(unipool_ctx* ctx, const ExpertBwdArgs& a, cudaStream_t s) {
