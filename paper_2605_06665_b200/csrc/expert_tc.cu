@@ -742,8 +742,8 @@ wgrad_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 
   // Ragged groups: the contraction length of a tile is its expert's row count over all layers.  The
   // experts are taken in order of decreasing length (ties by index) and dealt to the CTA pairs
-  // boustrophedon-wise (round 0: pair 0 .. P-1, round 1: pair P-1 .. 0, ...), so that every round holds
-  // tiles of similar size, the long ones come first, and no pair collects the longest tile of every round.
+  // boustrophedon-wise (first deal: pair 0 .. P-1, second deal: pair P-1 .. 0, ...), so that every deal holds
+  // tiles of similar size, the long ones come first, and no pair collects the longest tile of every deal.
   uint16_t* order = reinterpret_cast<uint16_t*>(smem + kBarOffset + 512);   // [n_experts] i-th longest expert
   int* kb_of = reinterpret_cast<int*>(smem + kPairStages * kPairStageBytes);  // scratch in the (still idle) staging tiles
   for (int e = threadIdx.x; e < p.n_experts; e += blockDim.x) kb_of[e] = wgrad_kblocks(p, e);
