@@ -263,17 +263,19 @@ struct ChunkCursor {
 
 // Epilogue of the gate/up projection for one warp's 32 rows: G and U leave TMEM, A = silu(G) * U is
 // formed, and the three bf16 chunks are staged and stored (GU through tmC0, A through tmC1).
-// Warps that share a TMEM lane quarter split the chunks: this warp takes ch0, ch0 + step, ...
+// t_g / t_u: TMEM addresses of this warp's lanes at the first G and the first U column; the chunks are
+// nch steps of 32 features from feat0.  Warps that share a TMEM lane quarter split the chunks: this
+// warp takes ch0, ch0 + step, ...
 __device__ __forceinline__ void epilogue_swiglu(const CUtensorMap* tmC0, const CUtensorMap* tmC1, const GemmParams& p,
-                                                uint32_t t_row, int nt, int row0, uint8_t* stg, int lane,
-                                                int ch0 = 0, int step = 1) {
+                                                uint32_t t_g, uint32_t t_u, int feat0, int nch, int row0, uint8_t* stg,
+                                                int lane, int ch0 = 0, int step = 1) {
 #pragma unroll 1
-  for (int ch = ch0; ch < BN / 2 / kChunk; ch += step) {
-    const int feat = nt * (BN / 2) + ch * kChunk;
+  for (int ch = ch0; ch < nch; ch += step) {
+    const int feat = feat0 + ch * kChunk;
     if (feat >= p.f) break;
     uint32_t rg[32], ru[32];
-    tc::tmem_ld_32x32(t_row + ch * kChunk, rg);
-    tc::tmem_ld_32x32(t_row + BN / 2 + ch * kChunk, ru);
+    tc::tmem_ld_32x32(t_g + ch * kChunk, rg);
+    tc::tmem_ld_32x32(t_u + ch * kChunk, ru);
     tc::tmem_ld_wait();
     float g[32], u[32], a[32];
 #pragma unroll
@@ -592,7 +594,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
       const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * BN;
 
       if constexpr (MODE == kFwd1) {
-        epilogue_swiglu(&tmC0, &tmC1, p, t_row, c.nt, row0, stg, lane);
+        epilogue_swiglu(&tmC0, &tmC1, p, t_row, t_row + BN / 2, c.nt * (BN / 2), BN / 2 / kChunk, row0, stg, lane);
       } else if constexpr (MODE == kFwd2 || MODE == kDgrad2) {
         epilogue_rows<MODE>(&tmC0, p, t_row, c.col0, c.ncols, row0, stg, lane, gchunk);
       } else if constexpr (MODE == kDgrad1) {
@@ -961,27 +963,29 @@ int map_chunk(const unipool_ctx* ctx, CUtensorMap* out, const void* base, uint64
 }
 
 // ---------------------------------------------------------------- row-tile GEMMs on CTA pairs
-// The forward GEMMs and the second dgrad at small groups are bound by what the SMs can pull in: a
-// 128 x 256 tile takes 48 KB of operands per k-block, most of it the expert's weights, which the
-// other row tiles of the same expert fetch again.  Here two row tiles of ONE expert share a CTA pair:
-// one tcgen05.mma.cta_group::2 of M = 256 (128 rows per CTA, each in its own TMEM) and N = 256, each
-// CTA loading its own 128 rows of A and HALF of the expert's 256 weight rows (B), 32 KB per k-block
-// and CTA, six stages.  A group with an odd number of row tiles ends in a pair whose second CTA has
-// no rows: it still supplies its half of B, loads no A, and stores nothing.  Scheduling, barriers and
-// commits follow the weight-gradient pair kernel above; the epilogues are the single-CTA ones.
+// A 128 x 256 tile takes 48 KB of operands per k-block, most of it the expert's weights, which the
+// other row tiles of the same expert fetch again, and an SM cannot pull more than ~100 GB/s out of
+// L2.  Here two row tiles of ONE expert share a CTA pair: one tcgen05.mma.cta_group::2 of M = 256
+// (128 rows per CTA, each in its own TMEM) and N = 256, each CTA loading its own 128 rows of A and
+// HALF of the expert's 256 weight rows (B), 32 KB per k-block and CTA, six stages.  The odd last tile
+// of a group is a half pair-tile: the M = 128 form of the same instruction, 64 rows per CTA (24 KB per
+// k-block and CTA).  Scheduling, barriers and commits follow the weight-gradient pair kernel above; the
+// epilogues are the single-CTA ones, addressed through the two accumulator layouts.
 // Six operand stages and four epilogue warps: a variant with eight epilogue warps (two per TMEM lane
-// quarter, taking alternate chunks; the helpers below support it) had to give one stage to their
-// staging tiles and was 8 - 12 % slower - the main loop lives on the bytes it keeps in flight.
+// quarter, taking alternate chunks) had to give one stage to their staging tiles and was 8 - 12 %
+// slower - the main loop lives on the bytes it keeps in flight.
 constexpr int kRowPairStages = 6;
 constexpr int kRowPairEpiWarps = 4;
 constexpr int kRowPairThreads = 64 + 32 * kRowPairEpiWarps;
 static_assert(kRowPairStages * kPairStageBytes + kRowPairEpiWarps * 8192 == kBarOffset, "shared-memory budget");
 
-struct PairTile { int e, mt, nt; bool mine, peer; };
+// half: the pair-tile is ONE row tile (the odd last tile of a group): each CTA takes 64 of its rows and the
+// MMA is the M = 128 form of cta_group::2.
+struct PairTile { int e, mt, nt; bool half; };
 
 // pair-tile q of the row space -> expert and first row tile; pp[e] = pair-tiles before expert e
 __device__ __forceinline__ PairTile pair_tile(const GemmParams& p, const uint16_t* pp, int tile, int n_nt,
-                                              int total_q, bool descending, int rank) {
+                                              int total_q, bool descending) {
   PairTile t;
   int q = tile / n_nt;
   t.nt = tile % n_nt;
@@ -994,17 +998,23 @@ __device__ __forceinline__ PairTile pair_tile(const GemmParams& p, const uint16_
   t.e = lo;
   const int first = p.group_offsets[lo] / BM, n_tiles = (p.group_offsets[lo + 1] - p.group_offsets[lo]) / BM;
   const int i = 2 * (q - (int)pp[lo]);
-  t.mt = first + i + rank;
-  t.mine = i + rank < n_tiles;
-  t.peer = i + (rank ^ 1) < n_tiles;
+  t.mt = first + i;
+  t.half = i + 1 >= n_tiles;
   return t;
 }
 
+// Accumulator layouts (read back with tcgen05.ld, lanes [32 w, 32 w + 32) for warp w of a CTA):
+//   M = 256: the CTA's 128 rows are lanes 0..127, the tile's 256 columns TMEM columns 0..255;
+//   M = 128: the CTA's 64 rows are lanes 0..63 for columns 0..127 AND lanes 64..127 for columns
+//            128..255, both at TMEM columns 0..127.
+// B halves: CTA r supplies columns [128 r, 128 r + 128) of the tile.  For the gate/up projection each
+// half is [64 gate features | the same 64 up features], so that G and U of one element meet in one
+// thread under both layouts.
 template <int MODE>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kRowPairThreads, 1)
-row_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                const __grid_constant__ CUtensorMap tmC0, const __grid_constant__ CUtensorMap tmC1,
-                const GemmParams p) {
+row_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmA64,
+                const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmC0,
+                const __grid_constant__ CUtensorMap tmC1, const GemmParams p) {
   static_assert(MODE == kFwd1 || MODE == kFwd2 || MODE == kDgrad2, "row tiles without epilogue operands");
   constexpr bool kBMn = Traits<MODE>::kBMn;
   constexpr bool kDescending = MODE == kFwd2 || MODE == kDgrad2;      // see tile_coord
@@ -1028,6 +1038,7 @@ row_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     *abort = 0;
     tc::fence_barrier_init();
     tc::tma_prefetch_desc(&tmA);
+    tc::tma_prefetch_desc(&tmA64);
     tc::tma_prefetch_desc(&tmB);
     tc::tma_prefetch_desc(&tmC0);
     if constexpr (MODE == kFwd1) tc::tma_prefetch_desc(&tmC1);
@@ -1036,10 +1047,11 @@ row_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     tc::tmem_alloc_pair(tmem_ptr, 512);
     tc::tmem_relinquish_pair();
   }
-  // pair-tiles before each expert: an expert of n row tiles takes ceil(n / 2)
+  // pair-tiles before each expert: an expert of n row tiles takes ceil(n / 2), the last one a half
+  // pair-tile when n is odd (part 1: floor(n / 2), the odd last tile is another kernel's)
   for (int e = threadIdx.x; e <= p.n_experts; e += blockDim.x) {
     int before = 0;
-    const int round_up = p.part == 1 ? 0 : 1;        // part 1: a group's odd last tile is another kernel's
+    const int round_up = p.part == 1 ? 0 : 1;
     for (int o = 0; o < e; ++o) before += ((p.group_offsets[o + 1] - p.group_offsets[o]) / BM + round_up) >> 1;
     pp[e] = (uint16_t)before;
   }
@@ -1062,19 +1074,25 @@ row_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       uint32_t phase = 0;
       bool ok = true;
       for (int tile = pair; tile < total && ok; tile += n_pairs) {
-        const PairTile t = pair_tile(p, pp, tile, n_nt, total_q, kDescending, rank);
+        const PairTile t = pair_tile(p, pp, tile, n_nt, total_q, kDescending);
         const int pe = p.expert_base + t.e;
-        const uint32_t tx = 2 * kPairHalfBytes + (t.mine ? kPairHalfBytes : 0) + (t.peer ? kPairHalfBytes : 0);
+        const uint32_t tx = 2 * (kPairHalfBytes + (t.half ? kPairHalfBytes / 2 : kPairHalfBytes));
         for (int kb = 0; kb < kblocks; ++kb) {
           if (!tc::mbar_wait(&empty_bar[stage], phase ^ 1u, abort)) { report_timeout(p, abort, 31); ok = false; break; }
           uint8_t* sA = smem + stage * kPairStageBytes;
           uint8_t* sB = sA + kPairHalfBytes;
           if (rank == 0) tc::mbar_expect_tx(&full_bar[stage], tx);              // both CTAs' bytes
-          if (t.mine) tc::tma_load_2d_pair(sA, &tmA, &full_bar[stage], kb * BK, t.mt * BM);
-          if constexpr (MODE == kFwd1) {           // B rows: 128 gate features (leader) or the same 128 up features
-            tc::tma_load_2d_pair(sB, &tmB, &full_bar[stage], kb * BK, pe * 2 * p.f + rank * p.f + t.nt * (BN / 2));
+          if (t.half) tc::tma_load_2d_pair(sA, &tmA64, &full_bar[stage], kb * BK, t.mt * BM + rank * (BM / 2));
+          else tc::tma_load_2d_pair(sA, &tmA, &full_bar[stage], kb * BK, (t.mt + rank) * BM);
+          if constexpr (MODE == kFwd1) {           // 64 gate features, then the same 64 up features
+            const int feat = t.nt * (BN / 2) + rank * 64;
+            tc::tma_load_2d_pair(sB, &tmB, &full_bar[stage], kb * BK, pe * 2 * p.f + feat);
+            tc::tma_load_2d_pair(sB + kMnBlockBytes, &tmB, &full_bar[stage], kb * BK, pe * 2 * p.f + p.f + feat);
           } else if constexpr (MODE == kFwd2) {
-            tc::tma_load_2d_pair(sB, &tmB, &full_bar[stage], kb * BK, pe * p.Ndim + t.nt * BN + rank * (BN / 2));
+#pragma unroll
+            for (int i = 0; i < 2; ++i)
+              tc::tma_load_2d_pair(sB + i * kMnBlockBytes, &tmB, &full_bar[stage], kb * BK,
+                                   pe * p.Ndim + t.nt * BN + rank * (BN / 2) + 64 * i);
           } else {
 #pragma unroll
             for (int i = 0; i < 2; ++i)
@@ -1090,7 +1108,8 @@ row_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer (leader CTA only)
     if (lane == 0 && rank == 0) {
-      constexpr uint32_t idesc = tc::instr_desc_bf16(BN, false, kBMn, 256);
+      constexpr uint32_t idesc_full = tc::instr_desc_bf16(BN, false, kBMn, 256);
+      constexpr uint32_t idesc_half = tc::instr_desc_bf16(BN, false, kBMn, 128);
       constexpr uint32_t b_lbo = kBMn ? kMnBlockBytes : 16;
       constexpr uint32_t a_step = 32 >> 4;                                   // K-major: 32 bytes per K = 16
       constexpr uint32_t b_step = (kBMn ? 16 * 128 : 32) >> 4;
@@ -1099,6 +1118,8 @@ row_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       int local = 0;
       bool ok = true;
       for (int tile = pair; tile < total && ok; tile += n_pairs) {
+        const PairTile t = pair_tile(p, pp, tile, n_nt, total_q, kDescending);
+        const uint32_t idesc = t.half ? idesc_half : idesc_full;
         const int acc = local & 1;
         const uint32_t acc_phase = (local >> 1) & 1;
         ++local;
@@ -1121,14 +1142,13 @@ row_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       }
     }
   } else {
-    // ------------------------------------------------------------ epilogue: this CTA's row tile
+    // ------------------------------------------------------------ epilogue: this CTA's rows of the pair-tile
     const int quarter = warp & 3;
-    const int half = (warp - 2) >> 2;                    // which of the quarter's two warps
     uint8_t* stg = smem + kRowPairStages * kPairStageBytes + (warp - 2) * 8192;
     int gchunk = 0, local = 0;
     (void)gchunk;
     for (int tile = pair; tile < total; tile += n_pairs) {
-      const PairTile t = pair_tile(p, pp, tile, n_nt, total_q, kDescending, rank);
+      const PairTile t = pair_tile(p, pp, tile, n_nt, total_q, kDescending);
       const int acc = local & 1;
       const uint32_t acc_phase = (local >> 1) & 1;
       ++local;
@@ -1137,12 +1157,24 @@ row_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         break;
       }
       tc::tc_fence_after_sync();
-      if (t.mine) {
-        const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * BN;
-        const int row0 = t.mt * BM + quarter * 32;
-        constexpr int kShare = kRowPairEpiWarps / 4;     // warps per TMEM lane quarter
-        if constexpr (MODE == kFwd1) epilogue_swiglu(&tmC0, &tmC1, p, t_row, t.nt, row0, stg, lane, half, kShare);
-        else epilogue_rows<MODE>(&tmC0, p, t_row, t.nt * BN, BN, row0, stg, lane, gchunk, half, kShare);
+      const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * BN;
+      if (!t.half) {
+        const int row0 = (t.mt + rank) * BM + quarter * 32;
+        if constexpr (MODE == kFwd1) {
+#pragma unroll 1
+          for (int h = 0; h < 2; ++h)                    // the two B halves: features [64 h, 64 h + 64) of the tile
+            epilogue_swiglu(&tmC0, &tmC1, p, t_row + 128 * h, t_row + 128 * h + 64, t.nt * (BN / 2) + 64 * h, 2, row0,
+                            stg, lane);
+        } else {
+          epilogue_rows<MODE>(&tmC0, p, t_row, t.nt * BN, BN, row0, stg, lane, gchunk);
+        }
+      } else {
+        const int h = quarter >> 1;                      // lanes 64..127 hold the second half of the columns
+        const int row0 = t.mt * BM + rank * (BM / 2) + (quarter & 1) * 32;
+        if constexpr (MODE == kFwd1)
+          epilogue_swiglu(&tmC0, &tmC1, p, t_row, t_row + 64, t.nt * (BN / 2) + 64 * h, 2, row0, stg, lane);
+        else
+          epilogue_rows<MODE>(&tmC0, p, t_row, t.nt * BN + 128 * h, BN / 2, row0, stg, lane, gchunk);
       }
       tc::tc_fence_before_sync();
       __syncwarp();
@@ -1177,34 +1209,35 @@ int launch(unipool_ctx* ctx, int phase, const CUtensorMap& tmA, const CUtensorMa
 
 // How the row-tile GEMMs (gate/up, down, second dgrad) of a call are scheduled:
 //   kRowsSingle  every tile on the single-CTA kernel;
-//   kRowsPairs   every tile on CTA pairs (a group of odd tile count ends in a half-empty pair);
+//   kRowsPairs   every tile on CTA pairs (the odd last tile of a group as a half pair-tile, M = 128);
 //   kRowsSplit   whole pairs on the pair kernel, then the odd last tiles on the single-CTA kernel.
-// Pairs move a third fewer operand bytes into the SMs.  Measured (interleaved runs, one B200): 10 %
-// faster per GEMM at 32 row tiles per group, no gain at 3 - 7 tiles, where the half-empty pairs cost
-// what the shared operand saves; the split schedule is 19 % SLOWER than single at 3 tiles per group
-// (the pair kernel's tiles of 12 k-blocks do not reach the single-CTA kernel's rate when most
-// operand bytes miss L2).  So: pairs when a batch of max_tokens gives the average expert eight row
-// tiles, single otherwise; UNIPOOL_ROW_PAIR = 0 / 1 / 2 forces single / pairs / split (a debugging
-// aid).  The pair schedule keeps 16-bit counts of pair-tiles.
+// Pairs move a third fewer operand bytes into the SMs.  Measured (interleaved runs, one B200), pairs
+// against single per GEMM: -10 % at 32 row tiles per group, -3 .. -8 % at 4 - 7 tiles, none at 2.7
+// tiles (341 rows), where two thirds of the operand bytes miss L2 and each k-block waits for the slower
+// of two CTAs' loads.  The split schedule streams every weight twice (once per kernel) and is 19 %
+// slower than single at 2.7 tiles.  So: pairs when a batch of max_tokens gives the average expert four
+// row tiles, single otherwise; UNIPOOL_ROW_PAIR = 0 / 1 / 2 forces single / pairs / split (a
+// debugging aid).  The pair schedule keeps 16-bit counts of pair-tiles.
 enum RowPlan { kRowsSingle = 0, kRowsPairs = 1, kRowsSplit = 2 };
 RowPlan row_plan(const unipool_ctx* ctx, int n_experts) {
   static const int forced = [] { const char* v = getenv("UNIPOOL_ROW_PAIR"); return v ? v[0] - '0' : -1; }();
   if (ctx->sm_count < 2 || ctx->row_capacity / (2 * BM) + n_experts >= 65535) return kRowsSingle;
   if (forced >= 0 && forced <= 2) return static_cast<RowPlan>(forced);
-  return (int64_t)ctx->cfg.max_tokens * ctx->cfg.top_k >= (int64_t)8 * BM * n_experts ? kRowsPairs : kRowsSingle;
+  return (int64_t)ctx->cfg.max_tokens * ctx->cfg.top_k >= (int64_t)4 * BM * n_experts ? kRowsPairs : kRowsSingle;
 }
 
-// One row-tile GEMM under `plan`.  tmB: the B map of the single-CTA kernel, tmBp: that of the pair kernel.
+// One row-tile GEMM under `plan`.  tmA / tmB: the operand maps of the single-CTA kernel; tmA64 / tmBp:
+// those of the pair kernel's half pair-tiles (64-row boxes of A) and of its B halves (64-row boxes).
 template <int MODE>
-int launch_rows(unipool_ctx* ctx, int phase, RowPlan plan, const CUtensorMap& tmA, const CUtensorMap& tmB,
-                const CUtensorMap& tmBp, const CUtensorMap& tmC0, const CUtensorMap& tmC1, GemmParams p,
-                cudaStream_t s) {
+int launch_rows(unipool_ctx* ctx, int phase, RowPlan plan, const CUtensorMap& tmA, const CUtensorMap& tmA64,
+                const CUtensorMap& tmB, const CUtensorMap& tmBp, const CUtensorMap& tmC0, const CUtensorMap& tmC1,
+                GemmParams p, cudaStream_t s) {
   PhaseTimer pt(ctx, phase, plan == kRowsSplit ? 2 : 1, s);
   if (plan != kRowsSingle) {
     p.part = plan == kRowsSplit ? 1 : 0;
     auto kern = row_pair_kernel<MODE>;
     UP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPairSmemTotal));
-    kern<<<ctx->sm_count / 2 * 2, kRowPairThreads, kPairSmemTotal, s>>>(tmA, tmBp, tmC0, tmC1, p);
+    kern<<<ctx->sm_count / 2 * 2, kRowPairThreads, kPairSmemTotal, s>>>(tmA, tmA64, tmBp, tmC0, tmC1, p);
     UP_LAUNCH_CHECK();
   }
   if (plan != kRowsPairs) {
@@ -1289,13 +1322,14 @@ int expert_fwd_tc(unipool_ctx* ctx, const ExpertFwdArgs& a, cudaStream_t s) {
   p.status = ctx->ws.status;
   p.group_offsets = a.offsets;
   const RowPlan plan = row_plan(ctx, a.n_experts);
-  CUtensorMap tmA, tmB, tmBp, tmC0, tmC1;
+  CUtensorMap tmA, tmA64, tmB, tmBp, tmC0, tmC1;
   int rc;
   // GU = Xp [W_gate; W_up]^T with the SwiGLU epilogue.  B tile = 128 gate rows + 128 up rows of the
   // same features, fetched as one 3-D box over W_gu viewed as [2M, f, d] (CTA pairs: one half each,
   // 128 rows of W_gu viewed as [2M f, d]).
   if ((rc = map_2d(ctx, &tmA, a.Xp, d, cap, 64, BM)) != UNIPOOL_OK) return rc;
-  if ((rc = map_2d(ctx, &tmBp, a.W_gu, d, (uint64_t)M * 2 * f, 64, BN / 2)) != UNIPOOL_OK) return rc;
+  if ((rc = map_2d(ctx, &tmA64, a.Xp, d, cap, 64, 64)) != UNIPOOL_OK) return rc;
+  if ((rc = map_2d(ctx, &tmBp, a.W_gu, d, (uint64_t)M * 2 * f, 64, 64)) != UNIPOOL_OK) return rc;
   {
     const uint64_t dims[3] = {(uint64_t)d, (uint64_t)f, (uint64_t)2 * M};
     const uint64_t strides[2] = {(uint64_t)d, (uint64_t)f * d};
@@ -1305,16 +1339,17 @@ int expert_fwd_tc(unipool_ctx* ctx, const ExpertFwdArgs& a, cudaStream_t s) {
   if ((rc = map_chunk(ctx, &tmC0, a.GU, 2 * f, cap, kMapBf16Chunk)) != UNIPOOL_OK) return rc;
   if ((rc = map_chunk(ctx, &tmC1, a.A, f, cap, kMapBf16Chunk)) != UNIPOOL_OK) return rc;
   p.Ndim = f; p.Kdim = d;
-  if ((rc = launch_rows<kFwd1>(ctx, UNIPOOL_PH_EXPERT_FWD_GU, plan, tmA, tmB, tmBp, tmC0, tmC1, p, s)) != UNIPOOL_OK)
+  if ((rc = launch_rows<kFwd1>(ctx, UNIPOOL_PH_EXPERT_FWD_GU, plan, tmA, tmA64, tmB, tmBp, tmC0, tmC1, p, s)) != UNIPOOL_OK)
     return rc;
   // Yp = A W_down^T
   if ((rc = map_2d(ctx, &tmA, a.A, f, cap, 64, BM)) != UNIPOOL_OK) return rc;
+  if ((rc = map_2d(ctx, &tmA64, a.A, f, cap, 64, 64)) != UNIPOOL_OK) return rc;
   if ((rc = map_2d(ctx, &tmB, a.W_down, f, (uint64_t)M * d, 64, BN)) != UNIPOOL_OK) return rc;
-  if ((rc = map_2d(ctx, &tmBp, a.W_down, f, (uint64_t)M * d, 64, BN / 2)) != UNIPOOL_OK) return rc;
-  if ((rc = map_2d(ctx, &tmC1, a.W_down, f, (uint64_t)M * d, 64, 64)) != UNIPOOL_OK) return rc;   // column slices
+  if ((rc = map_2d(ctx, &tmBp, a.W_down, f, (uint64_t)M * d, 64, 64)) != UNIPOOL_OK) return rc;   // 64-row boxes
+  tmC1 = tmBp;                                                                                    // column slices
   if ((rc = map_chunk(ctx, &tmC0, a.Yp, d, cap, kMapBf16Chunk)) != UNIPOOL_OK) return rc;
   p.Ndim = d; p.Kdim = f;
-  return launch_rows<kFwd2>(ctx, UNIPOOL_PH_EXPERT_FWD_DOWN, plan, tmA, tmB, tmBp, tmC0, tmC1, p, s);
+  return launch_rows<kFwd2>(ctx, UNIPOOL_PH_EXPERT_FWD_DOWN, plan, tmA, tmA64, tmB, tmBp, tmC0, tmC1, p, s);
 }
 
 int expert_bwd_tc(unipool_ctx* ctx, const ExpertBwdArgs& a, cudaStream_t s) {
@@ -1342,7 +1377,9 @@ int expert_bwd_tc(unipool_ctx* ctx, const ExpertBwdArgs& a, cudaStream_t s) {
   if ((rc = map_chunk(ctx, &tmC0, a.dXp, d, cap, kMapBf16Chunk)) != UNIPOOL_OK) return rc;
   p.Ndim = d; p.Kdim = 2 * f; p.overwrite = 1;
   p.group_offsets = a.offsets;
-  rc = launch_rows<kDgrad2>(ctx, UNIPOOL_PH_DGRAD_GU, row_plan(ctx, a.n_experts), tmA, tmB, tmB, tmC0, tmC0, p, s);
+  CUtensorMap tmA64;
+  if ((rc = map_2d(ctx, &tmA64, a.dGU, 2 * f, cap, 64, 64)) != UNIPOOL_OK) return rc;
+  rc = launch_rows<kDgrad2>(ctx, UNIPOOL_PH_DGRAD_GU, row_plan(ctx, a.n_experts), tmA, tmA64, tmB, tmB, tmC0, tmC0, p, s);
   if (rc != UNIPOOL_OK) return rc;
   if (a.wgrad) {
     PoolWgradArgs w{1, 0, a.offsets, a.Xp, a.A, a.dYp, a.dGU, a.expert_base, a.n_experts, a.dW_gu, a.dW_down,

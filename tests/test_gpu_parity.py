@@ -192,9 +192,10 @@ def test_softmax_router_mode(kw, T):
 
 @pytest.mark.parametrize("plan", ["1", "2"])
 def test_forced_row_gemm_schedules(plan):
-    """The row-tile GEMMs' other schedules (UNIPOOL_ROW_PAIR=1: every tile on CTA pairs, =2: whole
-    pairs on the pair kernel and the odd last tiles on the single-CTA kernel) pass the same bf16
-    parity cases; the switch is read once per process, so the cases run in a child process."""
+    """The row-tile GEMMs' other schedules (UNIPOOL_ROW_PAIR=1: every tile on CTA pairs, a group's odd
+    last tile as a half pair-tile; =2: whole pairs on the pair kernel and the odd last tiles on the
+    single-CTA kernel) pass the same bf16 parity cases; the switch is read once per process, so the
+    cases run in a child process."""
     import os
     import subprocess
     import sys
