@@ -30,8 +30,8 @@ if ROOT not in sys.path:
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of a workload's dominant kernel,
 # from the ncu capture summarised in profiles/grouped_gemm_182m_slice_ncu.txt: the 182m_slice case (a quarter
-# of the experts and of the rows of one 182m layer) moved 165.6 + 79.2 MB; a full launch is four times that.
-NCU_TRAFFIC = {("182m", "expert_fwd_gu"): 4 * (165.58e6 + 79.21e6)}
+# of the experts and of the rows of one 182m layer) moved 165.6 + 78.6 MB; a full launch is four times that.
+NCU_TRAFFIC = {("182m", "expert_fwd_gu"): 4 * (165.59e6 + 78.63e6)}
 
 METRIC = "moe_layer_fwd_bwd_tokens_per_s"
 UNIT = "tokens/s"
