@@ -360,8 +360,9 @@ route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   }
 }
 
-// dz of the router's derivative as bf16 [T, Mp] (columns >= M are zero); four lanes per token.
-template <bool SOFTMAX>
+// dz of the router's derivative as bf16 [T, Mp] (columns >= M are zero); four lanes per token, each
+// taking four neighbouring experts per step when the rows are 16-byte aligned (M % 4 == 0).
+template <bool SOFTMAX, int KT>
 __global__ void __launch_bounds__(256)
 router_dz16_kernel(const float* __restrict__ z, const float* __restrict__ znorm, const int32_t* __restrict__ idx,
                    const float* __restrict__ dgate, const float* __restrict__ coef, int T, int M, int Mp, int k,
@@ -372,39 +373,59 @@ router_dz16_kernel(const float* __restrict__ z, const float* __restrict__ znorm,
   const bool live = (gid >> 2) < T;
   const int t = live ? gid >> 2 : T - 1;
   const float* zr = z + (int64_t)t * M;
-  int e_sel[UNIPOOL_MAX_TOPK];
-  float dg_sel[UNIPOOL_MAX_TOPK];
+  int e_sel[KT];
+  float dg_sel[KT];
 #pragma unroll
-  for (int j = 0; j < UNIPOOL_MAX_TOPK; ++j) {
+  for (int j = 0; j < KT; ++j) {
     e_sel[j] = j < k ? idx[(int64_t)t * k + j] : -1;
     dg_sel[j] = j < k ? dgate[(int64_t)t * k + j] : 0.f;
   }
   auto ds_of = [&](int i) {
     float ds = coef ? __ldg(coef + i) : 0.f;
 #pragma unroll
-    for (int j = 0; j < UNIPOOL_MAX_TOPK; ++j)
+    for (int j = 0; j < KT; ++j)
       if (e_sel[j] == i) ds += dg_sel[j];
     return ds;
   };
   const float n = znorm[t];                       // ||z||; softmax: log sum exp(z)
+  const bool vec = (M & 3) == 0;
   float q = 0.f;
-  for (int i = sub; i < M; i += 4) q = fmaf(ds_of(i), SOFTMAX ? expf(zr[i] - n) : fmaxf(zr[i], 0.f), q);
+  if (vec) {
+    for (int i = 4 * sub; i < M; i += 16) {
+      const float4 zv = *reinterpret_cast<const float4*>(zr + i);
+      const float zz[4] = {zv.x, zv.y, zv.z, zv.w};
+#pragma unroll
+      for (int u = 0; u < 4; ++u) q = fmaf(ds_of(i + u), SOFTMAX ? expf(zz[u] - n) : fmaxf(zz[u], 0.f), q);
+    }
+  } else {
+    for (int i = sub; i < M; i += 4) q = fmaf(ds_of(i), SOFTMAX ? expf(zr[i] - n) : fmaxf(zr[i], 0.f), q);
+  }
   q += __shfl_xor_sync(0xffffffffu, q, 1);
   q += __shfl_xor_sync(0xffffffffu, q, 2);
   const float ne = n + eps;
   const float scale = sigma * c;
   const float qn = n > 0.f ? q / (n * ne * ne) : 0.f;
+  auto dz_of = [&](int i, float zi) {
+    if (SOFTMAX) return expf(zi - n) * (ds_of(i) - q);
+    return n > 0.f ? scale * ((zi > 0.f ? ds_of(i) / ne : 0.f) - zi * qn) : 0.f;
+  };
   if (live) {
     __nv_bfloat16* out = dz16 + (int64_t)t * Mp;
-    for (int i = sub; i < Mp; i += 4) {
-      float v = 0.f;
-      if (SOFTMAX) {
-        if (i < M) v = expf(zr[i] - n) * (ds_of(i) - q);
-      } else if (i < M && n > 0.f) {
-        const float zi = zr[i];
-        v = scale * ((zi > 0.f ? ds_of(i) / ne : 0.f) - zi * qn);
+    if (vec) {                                     // Mp is a multiple of 64: rows of dz16 are 8-byte aligned
+      for (int i = 4 * sub; i < Mp; i += 16) {
+        float v[4] = {0.f, 0.f, 0.f, 0.f};
+        if (i < M) {
+          const float4 zv = *reinterpret_cast<const float4*>(zr + i);
+          v[0] = dz_of(i, zv.x); v[1] = dz_of(i + 1, zv.y); v[2] = dz_of(i + 2, zv.z); v[3] = dz_of(i + 3, zv.w);
+        }
+        const __nv_bfloat162 lo = __floats2bfloat162_rn(v[0], v[1]), hi = __floats2bfloat162_rn(v[2], v[3]);
+        uint2 w;
+        w.x = *reinterpret_cast<const uint32_t*>(&lo);
+        w.y = *reinterpret_cast<const uint32_t*>(&hi);
+        *reinterpret_cast<uint2*>(out + i) = w;
       }
-      out[i] = __float2bfloat16_rn(v);
+    } else {
+      for (int i = sub; i < Mp; i += 4) out[i] = __float2bfloat16_rn(i < M ? dz_of(i, zr[i]) : 0.f);
     }
   }
   float part = (live && sub == 0 && !SOFTMAX) ? c * q / ne : 0.f;
@@ -497,7 +518,9 @@ int route_bwd_tc_launch(unipool_ctx* ctx, const void* x, int T, const float* W_r
     PhaseTimer pt(ctx, UNIPOOL_PH_ROUTE_BWD_DZ, 2, s);
     if ((rc = router_split_launch(ctx, W_r, M, s)) != UNIPOOL_OK) return rc;   // term 0 = bf16(W_r)
     const int64_t threads = (int64_t)T * 4;
-    auto kern = ctx->cfg.router_mode == UNIPOOL_ROUTER_SOFTMAX ? router_dz16_kernel<true> : router_dz16_kernel<false>;
+    const bool softmax = ctx->cfg.router_mode == UNIPOOL_ROUTER_SOFTMAX;
+    auto kern = k <= 2 ? (softmax ? router_dz16_kernel<true, 2> : router_dz16_kernel<false, 2>)
+                       : (softmax ? router_dz16_kernel<true, UNIPOOL_MAX_TOPK> : router_dz16_kernel<false, UNIPOOL_MAX_TOPK>);
     kern<<<(int)((threads + 255) / 256), 256, 0, s>>>(
         z_saved, znorm, idx, dgate, coef, T, M, Mp, k, sigma, ctx->cfg.c, ctx->cfg.eps, dz16, dsigma,
         ctx->ws.dsigma_acc, ctx->ws.tickets + 1);
