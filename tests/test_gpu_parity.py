@@ -152,6 +152,7 @@ def test_tiny_fp32_layers():
     (dict(M=12, k=2, private=4, L=3), 200),          # layer-private layout (Eq. 1)
     (dict(M=33, k=3), 1),                            # a single token: most experts empty
     (dict(M=8, k=2, zipf_beta=3.0), 700),            # one giant group, several empty experts
+    (dict(M=512, k=8, d=64, f=64), 40),              # the largest pool and top-k, the smallest widths
 ])
 def test_small_fp32_shapes(kw, T):
     cfg = small_cfg(**kw)
@@ -163,6 +164,8 @@ def test_small_fp32_shapes(kw, T):
     (dict(dtype="bf16", d=128, f=128, M=384, k=8, zipf_beta=0.4), 600),
     (dict(dtype="bf16", d=256, f=256, M=12, k=2, private=4, L=3), 520),
     (dict(dtype="bf16", d=128, f=128, M=10, k=3), 333),     # logit rows that are not 16-byte aligned
+    (dict(dtype="bf16", d=64, f=64, M=512, k=8), 257),      # the largest pool and top-k, the smallest widths
+    (dict(dtype="bf16", d=128, f=192, M=16, k=2), 1),       # a single token
     # groups of several row tiles: the forward GEMMs and the second dgrad run on CTA pairs
     (dict(dtype="bf16", d=256, f=320, M=4, k=2, zipf_beta=1.0), 2100),   # skewed: odd and even tile counts, f % 128 = 64
     (dict(dtype="bf16", d=192, f=256, M=2, k=1), 2500),                  # d % 256 = 192: a clipped last column tile
