@@ -1,15 +1,20 @@
 // Grouped SwiGLU expert GEMMs on the 5th-generation tensor cores (tcgen05) for
 // bf16 storage with fp32 accumulation: forward (Eq. 2's e_i), dgrad and wgrad.
 //
-// One persistent, warp-specialised kernel template serves all six GEMMs:
+// Persistent, warp-specialised kernels, one CTA per SM:
 //   warp 0      TMA producer   (one lane issues cp.async.bulk.tensor loads)
 //   warp 1      MMA issuer     (one lane issues tcgen05.mma; owns the TMEM allocation)
-//   warps 2-5   epilogue       (tcgen05.ld from TMEM, fused element-wise math, global stores)
+//   warps 2-5   epilogue       (tcgen05.ld from TMEM, fused element-wise math, results staged in
+//                               shared memory and written by TMA stores / add-reduces)
 // Operand tiles are staged in shared memory with the 128-byte swizzle, accumulators
 // are double-buffered in TMEM so the epilogue of one tile overlaps the main loop of
 // the next.  The tile schedule is read from device memory (group offsets), so no call
 // synchronises the host.  Every mbarrier wait is bounded: on expiry the kernel records
 // UNIPOOL_ERR_TIMEOUT in the status word, all roles leave, TMEM is released.
+//   grouped_gemm_tc_kernel<MODE>  one CTA per 128 x 256 tile (cta_group::1), all six GEMMs
+//   wgrad_pair_kernel             the weight gradient on CTA pairs (cta_group::2, M = 256)
+//   row_pair_kernel<MODE>         gate/up, down and second dgrad on CTA pairs (M = 256, and M = 128
+//                                 for a group's odd last tile)
 #include <cuda.h>
 
 #include <cstdlib>
