@@ -237,6 +237,17 @@ def test_aux_loss_identities():
 
 
 # ---------------------------------------------------------------- softmax router (the paper's baseline router)
+def test_softmax_router_hand_example():
+    ex = json.load(open(GOLDEN))["softmax_router"]
+    z = np.array([ex["z"]])
+    s, lse = O.softmax_router_scores(z)
+    np.testing.assert_allclose(s[0], ex["s"], rtol=1e-14)
+    assert lse[0] == pytest.approx(ex["lse"], rel=1e-14)
+    r = O.route(np.eye(3)[:1], np.zeros((3, 3)), 1.0, 1.0, 1e-6, 2, bias=z[0], mode="softmax")
+    assert r["idx"][0].tolist() == ex["top2"]
+    np.testing.assert_allclose(r["g"][0], ex["gates"], rtol=1e-14)
+
+
 def test_softmax_router_against_library_and_closed_forms():
     from scipy.special import logsumexp, softmax
     rng = np.random.default_rng(5)
