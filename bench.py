@@ -119,9 +119,15 @@ def algorithmic_bytes(cfg, cap_rows):
     T, d, k, m = cfg["T"], cfg["d"], cfg["k"], (cfg["private"] or cfg["M"])
     R = T * k
     b = 2
+    if cfg["dtype"] == "bf16":
+        # tensor-core router: "route_logits" is the split of W_r into bf16 terms (a few hundred KB, no
+        # bandwidth figure), "route_select" the fused kernel that reads x, writes the logits and does
+        # scoring, top-k and statistics
+        route = {"route_select": T * d * b + T * m * 4 + T * k * 8 + T * 4 + 3 * m * d * 2}
+    else:
+        route = {"route_logits": T * d * 4 + T * m * 4 + m * d * 4, "route_select": T * m * 4 + T * k * 8 + T * 4}
     return {
-        "route_logits": T * d * b + T * m * 4 + m * d * 4,
-        "route_select": T * m * 4 + T * k * 8 + T * 4,
+        **route,
         "dispatch_gather": T * d * b + R * d * b + R * 4,
         "combine": R * d * b + 2 * T * d * b + T * k * 8,
         "bwd_scale_gather": T * d * b + 2 * R * d * b + T * k * 12,     # dy + Yp read, dYp written, dgate
