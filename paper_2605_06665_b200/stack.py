@@ -259,24 +259,36 @@ class UniPoolStack:
             cur.wait_stream(side)
         return dx0
 
-    def accumulate_microbatches(self, batches, fbar0=None, T=None):
+    def accumulate_microbatches(self, batches, fbar0=None, T=None, exchange=None):
         """One optimizer step's worth of the path (App. D, App. G): every micro-batch (x0, upstream)
         runs forward, balance loss and backward; all of them add into the same gradient buffers (the
         first one overwrites them), and the balance loss of a micro-batch uses the token fractions
         f-bar of the PREVIOUS micro-batch - ``fbar0`` for the first (default: the f-bar this stack saw
-        last, or uniform 1/m).  Returns the per-micro-batch losses (device tensors)."""
+        last, or uniform 1/m).  Returns the per-micro-batch losses (device tensors).
+        With ``exchange`` (data-parallel replicas): f-bar of a micro-batch is summed over the
+        replicas (each replica's part is its counts over the whole batch's assignments) while its
+        backward pass runs - the lagged scheme needs no statistic of the current micro-batch, so no
+        reduction sits between forward and backward -, each loss returned is this
+        replica's share of the whole batch's (they add up over the replicas), and the gradients are
+        summed over the replicas once, after the last micro-batch."""
         if fbar0 is not None:
             self.fbar_lag = fbar0.to(self.device, torch.float32).reshape(self.fbar.shape).clone()
         elif self.fbar_lag is None:
             self.fbar_lag = torch.full_like(self.fbar, 1.0 / self.m)
         losses = []
         self.zero_router_grad()
+        replicas = 1 if exchange is None else exchange.world
+        n = len(batches)
         for i, (x0, upstream) in enumerate(batches):
             self.forward(x0, T)
-            self.aux_loss(T, fbar_prev=self.fbar_lag)
+            if exchange is not None:
+                exchange.finish()                      # the previous micro-batch's f-bar has arrived
+            self.aux_loss(T, fbar_prev=self.fbar_lag, replicas=replicas)
             losses.append(self.loss.clone())
             self.fbar_lag.copy_(self.fbar)             # updated after all layers finished forward, no gradient
-            self.backward(upstream, T, accumulate=i > 0)
+            if exchange is not None:
+                exchange.launch([self.fbar_lag])
+            self.backward(upstream, T, accumulate=i > 0, exchange=exchange if i == n - 1 else None)
         return losses
 
     def capture_step(self, x0=None, upstream=None, accumulate=True, out=None):

@@ -337,6 +337,33 @@ def test_single_replica_exchange_step_is_the_plain_step():
         st.close()
 
 
+def test_microbatches_with_single_replica_exchange():
+    """Micro-batch accumulation through the data-parallel exchange with one replica (every collective
+    the identity) reproduces the plain accumulation: losses and f-bar bit for bit, the gradients up to
+    the order of the fp32 add-reduces of the later micro-batches."""
+    import torch
+    from paper_2605_06665_b200 import dp
+    cfg = small_cfg(dtype="bf16", d=256, f=384, M=16, k=2, L=3)
+    T = 500
+    batches = []
+    for seed in (20, 21, 22):
+        inp = synth.make_inputs(cfg, seed=seed, T=T)
+        batches.append((torch.from_numpy(inp["x0"]).cuda().bfloat16(), torch.from_numpy(inp["upstream"]).cuda().bfloat16()))
+    inputs = synth.make_inputs(cfg, seed=20, T=T)
+    results = []
+    for exchange in (None, dp.GradientExchange(1)):
+        st = build_stack(cfg, inputs, T=T, deferred_wgrad=True)
+        losses = st.accumulate_microbatches(batches, exchange=exchange)
+        torch.cuda.synchronize()
+        st.ctx.check_status()
+        results.append([t.clone() for t in (st.dW_gu, st.dW_down, st.dW_r, st.fbar_lag, torch.stack(losses))])
+        st.close()
+    for a, b in zip(results[0][:3], results[1][:3]):
+        assert rel_max(to_np(b), to_np(a)) < 1e-6
+    for a, b in zip(results[0][3:], results[1][3:]):
+        assert torch.equal(a, b)
+
+
 def test_host_resident_step_matches_device_resident_step():
     """Inputs in pinned host memory (upstream copied in during the forward pass, x_L copied out during
     the backward pass, on a second stream) give the same step, eagerly and from a CUDA graph."""

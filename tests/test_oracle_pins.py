@@ -439,6 +439,29 @@ def test_data_parallel_replicas_sum_to_the_whole_batch():
     np.testing.assert_allclose(np.concatenate([r["dx0"] for r in reps]), whole["dx0"], rtol=1e-10, atol=1e-13)
 
 
+def test_data_parallel_replicas_with_one_step_behind_fbar():
+    """With the lagged f-bar (App. G) a replica needs no statistic of the other replicas for the current
+    micro-batch: its loss share (own score sums over the whole batch's token count) and its gradients
+    add up, over the replicas, to the whole batch's."""
+    pool, routers, x0, up, views = tiny_problem(seed=31, L=3, M=6, d=8, f=5, k=2, T=12)
+    k, c, eps, alpha = 2, 1.7, 1e-6, 0.3
+    fbar_prev = np.random.default_rng(1).dirichlet(np.ones(6))
+    whole = O.stack_objective_and_grads(x0, routers, pool, k, c, eps, alpha, up, fbar_prev=fbar_prev)
+    reps = [O.stack_objective_and_grads(x0[s], routers, pool, k, c, eps, alpha, up[s], fbar_prev=fbar_prev,
+                                        replica_stats=lambda cn, S: (cn, S, 12)) for s in (slice(0, 6), slice(6, 12))]
+    assert reps[0]["loss_aux"] + reps[1]["loss_aux"] == pytest.approx(whole["loss_aux"], rel=1e-13)
+    for name in ("W_gate", "W_up", "W_down"):
+        np.testing.assert_allclose(reps[0]["pool_grad"][name] + reps[1]["pool_grad"][name],
+                                   whole["pool_grad"][name], rtol=1e-9, atol=1e-12)
+    for l in range(3):
+        np.testing.assert_allclose(reps[0]["router_grads"][l]["dW_r"] + reps[1]["router_grads"][l]["dW_r"],
+                                   whole["router_grads"][l]["dW_r"], rtol=1e-9, atol=1e-12)
+    # the next micro-batch's f-bar is the sum of the replicas' counts over the whole batch's assignments
+    fb = sum(r["counts"].sum(0) for r in reps) / (3 * 12 * k)
+    np.testing.assert_allclose(fb, whole["counts"].sum(0) / (3 * 12 * k))
+    assert fb.sum() == pytest.approx(1.0)
+
+
 def test_unique_expert_accounting():
     """App. E: private experts give U = L exactly for top-1 (L k for top-k); a shared pool gives
     1 <= U <= min(M, L k); a hand case; and U equals the row-wise count of a dense indicator matrix."""
