@@ -16,7 +16,7 @@ import numpy as np
 
 
 def topk_norm(x, k):
-    """|| top-k( ReLU(x / ||x||_2) ) ||_2 for each row of x [m,E] (the loop body of Alg. 1)."""
+    """|| top-k( ReLU(x / ||x||_2) ) ||_2 for each row of x [m,E] (Alg. 1, App. H)."""
     y = np.maximum(x / np.linalg.norm(x, axis=1, keepdims=True), 0.0)
     y_sorted = -np.sort(-y, axis=1)               # descending
     top = y_sorted[:, :k]

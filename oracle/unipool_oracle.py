@@ -57,8 +57,8 @@ def norm_router_scores(z, sigma, c, eps):
 
 
 def softmax_router_scores(z):
-    """The conventional router the paper compares against (Sec. 4.3, first sentence; Sec. 5.1
-    "top-1 softmax routing"): s_i = exp(z_i) / sum_j exp(z_j) over the router's experts.
+    """The conventional router the paper compares against (Sec. 4.3, first sentence; the vanilla
+    baseline of Sec. 5.1): s_i = exp(z_i) / sum_j exp(z_j) over the router's experts.
 
     Returns (s [T,M], lse [T]) with lse = log sum_j exp(z_j); the largest logit is subtracted before
     exponentiation, which changes nothing in exact arithmetic.
@@ -71,9 +71,8 @@ def softmax_router_scores(z):
 
 
 def top_k(s, k):
-    """Indices of the k highest scores per token (Sec. 4.3, "top-k experts are
-    selected based on the highest scores"), descending score, ties broken by
-    the lowest expert index.  s [T,M] -> idx [T,k] int32.
+    """Indices of the k highest scores per token (Sec. 4.3, "Top-k selection"),
+    descending score, ties broken by the lowest expert index.  s [T,M] -> idx [T,k] int32.
     """
     # a stable sort of the negated scores keeps equal scores in index order
     order = np.argsort(-s, axis=-1, kind="stable")

@@ -13,6 +13,29 @@ def env_world():
             int(os.environ.get("LOCAL_RANK", "0")))
 
 
+def free_port():
+    """A TCP port that is free on 127.0.0.1 right now (for the ranks' rendezvous)."""
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return int(s.getsockname()[1])
+
+
+def launch_command(n_ranks, script, argv, port):
+    """The command that runs ``script argv`` as ``n_ranks`` processes of one node (one per GPU) under
+    ``torch.distributed.run``; the ranks meet on 127.0.0.1:``port``."""
+    import sys
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={int(n_ranks)}",
+            "--master-addr", "127.0.0.1", "--master-port", str(int(port)), script] + list(argv)
+
+
+def launch_ranks(n_ranks, script, argv, env=None):
+    """Starts the ranks (see ``launch_command``), waits for them and returns the launcher's exit code.
+    The children find RANK / LOCAL_RANK / WORLD_SIZE / MASTER_* in their environment."""
+    import subprocess
+    return subprocess.call(launch_command(n_ranks, script, argv, free_port()), env=env)
+
+
 def shard_seed(rank):
     """Seed of rank ``rank``'s synthetic token shard: every rank draws its own tokens."""
     return int(rank)

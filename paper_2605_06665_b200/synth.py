@@ -7,7 +7,9 @@ it.  The token values stand in for a training micro-batch (the paper trains on
 
 Recipe: x_0 ~ N(0,1) [T,d]; every expert and router weight ~ N(0, 0.02^2);
 sigma_l = 1; upstream gradient ~ N(0,1) [T,d]; one numpy PCG64 stream per tensor,
-derived from (seed, tensor tag, layer).  In bf16 mode every tensor is rounded to
+derived from (seed, tensor tag, layer) - for the pool weights one stream per
+(seed, tensor tag, expert), so that the experts of a large pool can be drawn side by
+side on all host cores.  In bf16 mode every tensor is rounded to
 a bf16-representable value once, here, and returned as float32, so that both
 sides read identical numbers.  The skewed workload adds to layer l's logits the
 bias  beta * (ln p(rank_l(i)) - mean_j ln p(j)),  p(r) ~ r^-1.1 (Zipf), rank_l a
@@ -19,6 +21,9 @@ has at least one expert without tokens (and one expert that more than 5 % of the
 tokens select).
 """
 from __future__ import annotations
+
+import os
+from concurrent.futures import ThreadPoolExecutor
 
 import numpy as np
 
@@ -38,10 +43,14 @@ CONFIGS = {
     "978m_vanilla":   dict(L=24, d=1536, f=4096, M=192, k=2, T=32768, dtype="bf16", private=8, zipf_beta=0.0),
     # a quarter of one 182m layer (same rows per expert, same tiles): small profiler captures
     "182m_slice":     dict(L=1,  d=768,  f=2048, M=24,  k=2, T=4096,  dtype="bf16", private=0, zipf_beta=0.0),
+    # profiler cases of the 978m shapes: an eighth of one layer (same rows per expert and tiles), and one
+    # layer's full token batch over an eighth of the pool (activations larger than the L2 cache)
+    "978m_slice":     dict(L=1,  d=1536, f=4096, M=24,  k=2, T=4096,  dtype="bf16", private=0, zipf_beta=0.0),
+    "978m_tokens":    dict(L=1,  d=1536, f=4096, M=24,  k=2, T=32768, dtype="bf16", private=0, zipf_beta=0.0),
     "fine_zipf":      dict(L=12, d=768,  f=512,  M=384, k=8, T=16384, dtype="bf16", private=0, zipf_beta=0.4),
 }
 
-EPS = 1e-6          # "small constant for numerical stability" of Eq. 7
+EPS = 1e-6          # epsilon of Eq. 7 (the paper gives no value)
 ALPHA = 1e-2        # balance-loss coefficient used at the 182M scale (App. D)
 INIT_STD = 0.02
 ZIPF_S = 1.1
@@ -65,6 +74,24 @@ def _normal(seed, tag, layer, shape, std, bf16):
     if std != 1.0:
         a *= np.float32(std)
     return round_to_bf16(a) if bf16 else a
+
+
+def _pool_tensor(seed, tag, shape, std, bf16):
+    """[M, rows, cols] pool weights, expert e from the stream (seed, tag, e); the experts are drawn,
+    scaled and rounded by a pool of host threads (numpy releases the interpreter lock meanwhile)."""
+    out = np.empty(shape, dtype=np.float32)
+
+    def fill(e):
+        out[e] = _normal(seed, tag, e, shape[1:], std, bf16)
+
+    workers = min(len(os.sched_getaffinity(0)), shape[0]) if hasattr(os, "sched_getaffinity") else 1
+    if workers <= 1:
+        for e in range(shape[0]):
+            fill(e)
+    else:
+        with ThreadPoolExecutor(max_workers=workers) as ex:
+            list(ex.map(fill, range(shape[0])))
+    return out
 
 
 def router_width(cfg):
@@ -108,9 +135,9 @@ def make_inputs(cfg, seed=0, T=None, L=None):
     bf16 = cfg["dtype"] == "bf16"
     m = router_width(cfg)
     pool = dict(
-        W_gate=_normal(seed, 1, 0, (M, f, d), INIT_STD, bf16),
-        W_up=_normal(seed, 2, 0, (M, f, d), INIT_STD, bf16),
-        W_down=_normal(seed, 3, 0, (M, d, f), INIT_STD, bf16),
+        W_gate=_pool_tensor(seed, 1, (M, f, d), INIT_STD, bf16),
+        W_up=_pool_tensor(seed, 2, (M, f, d), INIT_STD, bf16),
+        W_down=_pool_tensor(seed, 3, (M, d, f), INIT_STD, bf16),
     )
     routers = []
     for l in range(L):

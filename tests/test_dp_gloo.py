@@ -137,3 +137,38 @@ def test_single_rank_is_the_identity():
     assert t.tolist() == [0.0, 1.0, 2.0, 3.0]
     assert dp.max_over_ranks(3.5, 1) == 3.5
     assert dp.whole_job_throughput(100, 1, 10.0) == 1e4
+
+
+LAUNCHED = textwrap.dedent("""
+    import os, sys, json
+    sys.path.insert(0, %r)
+    import torch.distributed as dist
+    from paper_2605_06665_b200 import dp
+    world, rank, local = dp.env_world()
+    dist.init_process_group("gloo")
+    ms = dp.max_over_ranks(1.0 + rank, world)
+    with open(os.path.join(sys.argv[1], "rank%%d.json" %% rank), "w") as fh:
+        json.dump(dict(world=world, rank=rank, local=local, ms=ms, argv=sys.argv[2:]), fh)
+    dist.barrier()
+    dist.destroy_process_group()
+""" % ROOT)
+
+
+def test_launcher_starts_one_process_per_rank(tmp_path):
+    """`bench.py --gpus N` without a launcher's environment starts its ranks through dp.launch_ranks:
+    here a stub worker stands in for the benchmark (gloo, CPU)."""
+    import json
+    sys.path.insert(0, ROOT)
+    from paper_2605_06665_b200 import dp
+    script = tmp_path / "stub.py"
+    script.write_text(LAUNCHED)
+    cmd = dp.launch_command(2, str(script), ["x"], 12345)
+    assert cmd[1:3] == ["-m", "torch.distributed.run"] and "--nproc-per-node=2" in cmd
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1" and cmd[-2:] == [str(script), "x"]
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    rc = dp.launch_ranks(2, str(script), [str(tmp_path), "--steps", "3"], env=env)
+    assert rc == 0
+    got = [json.load(open(tmp_path / f"rank{r}.json")) for r in range(2)]
+    for r, g in enumerate(got):
+        assert g["world"] == 2 and g["rank"] == r and g["local"] == r
+        assert g["ms"] == 2.0 and g["argv"] == ["--steps", "3"]

@@ -14,6 +14,13 @@ Each layer's oracle consumes the GPU's own x_l and dx_{l+1} (converted to float6
 layer's arithmetic is compared: bf16 rounding of x_l legitimately re-routes a few tokens per layer.
 Tolerances as in the small-shape tests: 1e-2 of the largest reference magnitude for bf16 storage,
 1e-5 for the fp32 quantities of the router and the balance loss.
+
+The router, the maps and the balance loss are always evaluated in float64.  The expert path of the
+978M-shaped workloads is evaluated by the oracle in float32 (its arithmetic follows the dtype of its
+inputs): the sampled tokens of a layer touch every one of the 192 experts, and widening 14.5 GB of
+weights to float64 once per layer and pass would take the oracle minutes per layer.  The operands
+are bf16 values, so every product is exact in float32 and only the summation differs (relative
+1e-6 or so against a bound of 1e-2).
 """
 import numpy as np
 import pytest
@@ -25,7 +32,7 @@ from parity_utils import build_stack, check_routing, f64, rel_max, to_np
 pytestmark = pytest.mark.gpu
 
 TOL = 1e-2
-N_TOKENS = 192          # sampled tokens per layer
+N_TOKENS = 1024         # sampled tokens per layer
 N_EXPERTS = 3           # random experts on top of the three structural picks
 
 
@@ -44,7 +51,7 @@ def sampled_experts(total_counts, rng):
 @pytest.mark.parametrize("name,L", [
     ("182m", None), ("182m_vanilla", None), ("182m_pool40", None), ("fine_zipf", None),
     ("182m_vanilla_softmax", None),
-    ("978m", 2),            # full layer shape and pool; two layers keep the host-side set-up affordable
+    ("978m", None), ("978m_pool128", None), ("978m_vanilla", None),
 ])
 def test_full_size_sampled_parity(name, L):
     import torch
@@ -55,7 +62,8 @@ def test_full_size_sampled_parity(name, L):
     mode = cfg.get("router", "norm")
     inputs = synth.make_inputs(cfg, seed=0, L=L)
     st = build_stack(cfg, inputs, L=L, deferred_wgrad=True)
-    pool = inputs["pool"]                                   # float32 holding bf16 values; products run in float64
+    pool = inputs["pool"]                                   # float32 holding bf16 values
+    ex = f64 if d <= 768 else (lambda a: np.asarray(a, dtype=np.float32))   # dtype of the oracle's expert path
     routers = [dict(W_r=f64(r["W_r"]), sigma=float(r["sigma"]),
                     bias=None if r["bias"] is None else f64(r["bias"])) for r in inputs["routers"]]
     c, eps, alpha = st.c, synth.EPS, synth.ALPHA
@@ -85,9 +93,9 @@ def test_full_size_sampled_parity(name, L):
         tok_gpu = to_np(st.token_of[l])
         assert (tok_gpu[:used] == token_of).all() and (tok_gpu[used:] == -1).all()
         tokens = np.sort(rng.choice(T, size=N_TOKENS, replace=False))
-        y_ref = O.moe_layer_output(x_l, idx_gpu, ref["g"], pool, synth.expert_base(cfg, l), tokens=tokens)
+        y_ref = O.moe_layer_output(ex(x_l), idx_gpu, ex(ref["g"]), pool, synth.expert_base(cfg, l), tokens=tokens)
         got = f64(to_np(st.x[l + 1][torch.from_numpy(tokens).cuda()]))
-        assert rel_max(got, x_l[tokens] + y_ref) < TOL
+        assert rel_max(got, x_l[tokens] + f64(y_ref)) < TOL
         ref["tokens"] = tokens
         routes.append(ref)
 
@@ -119,7 +127,7 @@ def test_full_size_sampled_parity(name, L):
         for e in es:
             pe = synth.expert_base(cfg, l) + e
             for n in grad:
-                grad[n].setdefault(pe, np.zeros(pool[n].shape[1:], dtype=np.float64))
+                grad[n].setdefault(pe, np.zeros(pool[n].shape[1:], dtype=ex(0.0).dtype))
     st.dW_gu.fill_(3.0); st.dW_down.fill_(-5.0)               # the overwriting pass must replace these
     st.zero_router_grad()
     dx_cur = torch.from_numpy(inputs["upstream"]).to(st.device, st.tdtype)
@@ -131,14 +139,15 @@ def test_full_size_sampled_parity(name, L):
         base = synth.expert_base(cfg, l)
         dxn = f64(to_np(dx_cur))
         tokens = r["tokens"]
-        dx_e, dg = O.expert_path_backward(xs[l], r["idx"], r["g"], pool, dxn, base, tokens=tokens)
+        dx_e, dg = O.expert_path_backward(ex(xs[l]), r["idx"], ex(r["g"]), pool, ex(dxn), base, tokens=tokens)
+        dx_e, dg = f64(dx_e), f64(dg)
         assert rel_max(to_np(st.dgate)[tokens], dg) < TOL
         rb = O.route_backward(xs[l][tokens], routers[l]["W_r"], routers[l]["sigma"], c, eps, r["z"][tokens],
                               r["n"][tokens], r["idx"][tokens], dg, coefs[l], mode=mode)
         got = f64(to_np(dx_out[torch.from_numpy(tokens).cuda()]))
         assert rel_max(got, dxn[tokens] + dx_e + rb["dx"]) < TOL
         if l in experts:
-            O.expert_path_backward(xs[l], r["idx"], r["g"], pool, dxn, base, grad, experts=experts[l])
+            O.expert_path_backward(ex(xs[l]), r["idx"], ex(r["g"]), pool, ex(dxn), base, grad, experts=experts[l])
         dx_cur = dx_out
     if st.deferred_wgrad:
         from paper_2605_06665_b200 import binding as B
@@ -161,3 +170,5 @@ def test_full_size_sampled_parity(name, L):
         for e in untouched[:8]:
             assert not to_np(st.dW_gu[int(e)]).any() and not to_np(st.dW_down[int(e)]).any()
     st.close()
+    del st, dx_cur, dx_out
+    torch.cuda.empty_cache()                                 # the next workload needs the memory

@@ -120,11 +120,14 @@ def run_layer_checks(cfg, T, L, seed=0, zero_grad_check=True):
                               cc["idx"], dg, coefs[l], mode=mode)
         assert rel_max(to_np(dx_out), dxn + dx_e + rb["dx"]) < tol
         assert rel_max(to_np(st.dW_r[l]), rb["dW_r"]) < tol
-        # dsigma is a signed sum over all (token, expert) terms: the bound scales with the sum of
-        # their magnitudes, not with the (cancelling) total
-        ne = cc["n"] + eps
-        dsigma_scale = c * np.sum(np.abs(rb["ds"]) * np.maximum(cc["z"], 0.0) / ne[:, None])
-        assert abs(float(st.dsigma[l]) - rb["dsigma"]) <= tol * max(dsigma_scale, 1e-3)
+        if cfg["dtype"] == "fp32":
+            assert abs(float(st.dsigma[l]) - rb["dsigma"]) <= tol * max(abs(rb["dsigma"]), 1e-3)
+        else:
+            # dsigma is a signed sum over all (token, expert) terms whose inputs (dgate) carry bf16
+            # rounding: the bound scales with the sum of their magnitudes, not with the (cancelling) total
+            ne = cc["n"] + eps
+            dsigma_scale = c * np.sum(np.abs(rb["ds"]) * np.maximum(cc["z"], 0.0) / ne[:, None])
+            assert abs(float(st.dsigma[l]) - rb["dsigma"]) <= tol * max(dsigma_scale, 1e-3)
         dx_cur = dx_out
     f = cfg["f"]
     dW_gu = to_np(st.dW_gu)

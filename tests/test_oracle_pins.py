@@ -234,6 +234,14 @@ def test_aux_loss_identities():
     lo, fb_now, co = O.pool_aux_loss(counts, S, T, k, alpha, fbar_prev=prev)
     assert lo == pytest.approx(alpha * M * np.sum(prev * (S / T).mean(0)), rel=1e-13)
     np.testing.assert_allclose(fb_now, fbar)
+    # ... also in the gradient: with the lagged fbar held constant the loss is linear in the scores,
+    # d loss / d s^(l)_{t,i} = alpha M prev_i / (L T)  (App. G: only P carries gradient)
+    np.testing.assert_allclose(co, alpha * M * prev / (L * T), rtol=1e-14)
+    for (l, i) in [(1, 2), (2, 5)]:
+        S2 = S.copy()
+        S2[l, i] += dS
+        l2, _, _ = O.pool_aux_loss(counts, S2, T, k, alpha, fbar_prev=prev)
+        assert (l2 - lo) / dS == pytest.approx(co[i], rel=1e-8)
 
 
 # ---------------------------------------------------------------- softmax router (the paper's baseline router)
