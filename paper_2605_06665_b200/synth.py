@@ -5,7 +5,8 @@ method's arithmetic, so the CUDA path and the CPU oracle can both be fed from
 it.  The token values stand in for a training micro-batch (the paper trains on
 16 x 1024-token micro-batches, App. D): only shapes matter to the MoE layer.
 
-Recipe: x_0 ~ N(0,1) [T,d]; every expert and router weight ~ N(0, 0.02^2);
+Recipe: x_0 ~ N(0,1) [T,d]; every expert and router weight ~ N(0, 0.02^2) (the down projection of
+the 24-layer workloads ~ N(0, 0.02^2 / (2 L)), see CONFIGS);
 sigma_l = 1; upstream gradient ~ N(0,1) [T,d]; one numpy PCG64 stream per tensor,
 derived from (seed, tensor tag, layer) - for the pool weights one stream per
 (seed, tensor tag, expert), so that the experts of a large pool can be drawn side by
@@ -38,9 +39,16 @@ CONFIGS = {
     "182m_vanilla_softmax": dict(L=12, d=768, f=2048, M=96, k=1, T=16384, dtype="bf16", private=8, zipf_beta=0.0,
                                  router="softmax"),
     "182m_pool40":    dict(L=12, d=768,  f=2048, M=40,  k=2, T=16384, dtype="bf16", private=0, zipf_beta=0.0),
-    "978m":           dict(L=24, d=1536, f=4096, M=192, k=2, T=32768, dtype="bf16", private=0, zipf_beta=0.0),
-    "978m_pool128":   dict(L=24, d=1536, f=4096, M=128, k=2, T=32768, dtype="bf16", private=0, zipf_beta=0.0),
-    "978m_vanilla":   dict(L=24, d=1536, f=4096, M=192, k=2, T=32768, dtype="bf16", private=8, zipf_beta=0.0),
+    # 24 residual blocks without a normalisation layer between them: with W_down ~ N(0, 0.02^2) the
+    # stream grows quadratically per block, overflows bf16 near block 20 and the routing collapses onto
+    # two experts.  These workloads therefore draw W_down with the depth-scaled standard deviation
+    # 0.02 / sqrt(2 L) that transformer frameworks apply to output projections.
+    "978m":           dict(L=24, d=1536, f=4096, M=192, k=2, T=32768, dtype="bf16", private=0, zipf_beta=0.0,
+                           scaled_down_init=True),
+    "978m_pool128":   dict(L=24, d=1536, f=4096, M=128, k=2, T=32768, dtype="bf16", private=0, zipf_beta=0.0,
+                           scaled_down_init=True),
+    "978m_vanilla":   dict(L=24, d=1536, f=4096, M=192, k=2, T=32768, dtype="bf16", private=8, zipf_beta=0.0,
+                           scaled_down_init=True),
     # a quarter of one 182m layer (same rows per expert, same tiles): small profiler captures
     "182m_slice":     dict(L=1,  d=768,  f=2048, M=24,  k=2, T=4096,  dtype="bf16", private=0, zipf_beta=0.0),
     # profiler cases of the 978m shapes: an eighth of one layer (same rows per expert and tiles), and one
@@ -134,10 +142,11 @@ def make_inputs(cfg, seed=0, T=None, L=None):
     d, f, M = cfg["d"], cfg["f"], cfg["M"]
     bf16 = cfg["dtype"] == "bf16"
     m = router_width(cfg)
+    down_std = INIT_STD / float(np.sqrt(2.0 * cfg["L"])) if cfg.get("scaled_down_init") else INIT_STD
     pool = dict(
         W_gate=_pool_tensor(seed, 1, (M, f, d), INIT_STD, bf16),
         W_up=_pool_tensor(seed, 2, (M, f, d), INIT_STD, bf16),
-        W_down=_pool_tensor(seed, 3, (M, d, f), INIT_STD, bf16),
+        W_down=_pool_tensor(seed, 3, (M, d, f), down_std, bf16),
     )
     routers = []
     for l in range(L):

@@ -96,6 +96,11 @@ def test_full_size_sampled_parity(name, L):
         y_ref = O.moe_layer_output(ex(x_l), idx_gpu, ex(ref["g"]), pool, synth.expert_base(cfg, l), tokens=tokens)
         got = f64(to_np(st.x[l + 1][torch.from_numpy(tokens).cuda()]))
         assert rel_max(got, x_l[tokens] + f64(y_ref)) < TOL
+        # ... and at the scale of the expert outputs themselves (the residual stream can dwarf them): the
+        # gate-weighted sum of the GPU's un-combined expert rows of the sampled tokens
+        rows = torch.from_numpy(to_np(st.row_of[l])[tokens].astype(np.int64)).cuda()          # [n, k]
+        y_rows = f64(to_np(st.Yp[st.slot(l)][rows.reshape(-1)])).reshape(len(tokens), k, d)
+        assert rel_max(np.einsum("tj,tjd->td", f64(ref["g"])[tokens], y_rows), f64(y_ref)) < TOL
         ref["tokens"] = tokens
         routes.append(ref)
 
