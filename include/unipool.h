@@ -130,6 +130,17 @@ int unipool_route(unipool_ctx* ctx, const void* x, int32_t T, const float* W_r, 
                   int32_t* counts, float* score_sum, float* znorm, float* z_saved,
                   unipool_stream stream);
 
+/* Optional set-up of the routers of a bf16 context, once per parameter update.  unipool_route and
+ * unipool_route_bwd compute the fp32 logits of Eq. 7 on the tensor cores from three bf16 terms of the
+ * fp32 router weights (W = W0 + W1 + W2, every product exact in fp32).  Without this call each of them
+ * splits the W_r it is given on every call.  With it the terms of all n_layers routers
+ * (W_r [n_layers, n_experts, d], contiguous) are formed by one kernel and kept in the workspace: a
+ * later route / route_bwd call whose W_r points at one of these layers (W_r + l*n_experts*d) uses
+ * them.  They are a copy: call again after the weights change; n_layers = 0 forgets them.  A context
+ * of dtype UNIPOOL_FP32 ignores the call.  n_layers <= config.n_layers. */
+int unipool_router_prepare(unipool_ctx* ctx, const float* W_r, int32_t n_layers, int32_t n_experts,
+                           unipool_stream stream);
+
 /* Token permute into expert-contiguous order (the grouped layout behind
  * Table 7's "Grouped GEMM"; Eq. 2 evaluates every selected expert, nothing is
  * dropped).  Stable: rows of one expert keep token-major order.

@@ -25,7 +25,7 @@ EXPORTS = (
     "unipool_expert_fwd", "unipool_combine", "unipool_expert_bwd", "unipool_pool_wgrad",
     "unipool_pool_aux_loss", "unipool_route_bwd", "unipool_calibrate_c",
     "unipool_profile_enable", "unipool_profile_read", "unipool_dispatch_static",
-    "unipool_unique_experts",
+    "unipool_unique_experts", "unipool_router_prepare",
 )
 
 PHASES = (
@@ -79,6 +79,8 @@ def lib():
     L.unipool_check_status.argtypes = [vp, vp]
     L.unipool_route.restype = ctypes.c_int
     L.unipool_route.argtypes = [vp, vp, i32, vp, f32, vp, i32, vp, vp, vp, vp, vp, vp, vp]
+    L.unipool_router_prepare.restype = ctypes.c_int
+    L.unipool_router_prepare.argtypes = [vp, vp, i32, i32, vp]
     L.unipool_dispatch.restype = ctypes.c_int
     L.unipool_dispatch.argtypes = [vp, vp, i32, vp, i32, vp, vp, vp, vp, vp, vp]
     L.unipool_dispatch_static.restype = ctypes.c_int
@@ -179,6 +181,9 @@ class Context:
     def route(self, x, T, W_r, sigma, bias, n_experts, idx, gate, counts, score_sum, znorm, z_saved):
         _check(lib().unipool_route(self.handle, _p(x), T, _p(W_r), sigma, _p(bias), n_experts, _p(idx),
                                    _p(gate), _p(counts), _p(score_sum), _p(znorm), _p(z_saved), _stream()))
+
+    def router_prepare(self, W_r, n_layers, n_experts):
+        _check(lib().unipool_router_prepare(self.handle, _p(W_r), n_layers, n_experts, _stream()))
 
     def dispatch(self, x, T, idx, n_experts, offsets, row_of, token_of, tile_expert, Xp):
         _check(lib().unipool_dispatch(self.handle, _p(x), T, _p(idx), n_experts, _p(offsets), _p(row_of),

@@ -51,16 +51,17 @@ Workspace carve_workspace(const unipool_config& cfg, void* base) {
   w.route_sums = reinterpret_cast<double*>(take(UNIPOOL_MAX_EXPERTS * sizeof(double)));
   w.tickets = reinterpret_cast<uint32_t*>(take(8 * sizeof(uint32_t)));
   w.dsigma_acc = reinterpret_cast<double*>(take(2 * sizeof(double)));
-  w.split_any = reinterpret_cast<int32_t*>(take(4 * sizeof(int32_t)));
+  w.split_any = reinterpret_cast<int32_t*>(take((size_t)(cfg.n_layers + 1) * 4 * sizeof(int32_t)));
   w.block_hist = reinterpret_cast<int32_t*>(take((size_t)blocks * UNIPOOL_MAX_EXPERTS * sizeof(int32_t)));
   {
     const size_t mp = ((size_t)cfg.pool_size + 63) / 64 * 64;
     const size_t per_token = cfg.dtype == UNIPOOL_BF16 ? mp * 2 : (size_t)cfg.pool_size * sizeof(float);
     w.dz = reinterpret_cast<float*>(take((size_t)cfg.max_tokens * per_token));
   }
-  w.w_split = cfg.dtype == UNIPOOL_BF16 ? take((size_t)3 * cfg.pool_size * cfg.d_model * 2) : nullptr;
+  w.w_split = cfg.dtype == UNIPOOL_BF16
+                  ? take((size_t)(cfg.n_layers + 1) * 3 * cfg.pool_size * cfg.d_model * 2) : nullptr;
   {
-    const size_t tiles = ((size_t)cfg.max_tokens + 127) / 128;
+    const size_t tiles = 2 * (((size_t)cfg.max_tokens + 255) / 256);   // CTAs of the router: whole pairs
     w.part_counts = reinterpret_cast<int32_t*>(take(tiles * cfg.pool_size * sizeof(int32_t)));
     w.part_sums = reinterpret_cast<float*>(take(tiles * cfg.pool_size * sizeof(float)));
     w.part_dsigma = reinterpret_cast<float*>(take((((size_t)cfg.max_tokens + 63) / 64) * sizeof(float)));
@@ -142,6 +143,8 @@ int unipool_create(unipool_ctx** out, const unipool_config* cfg, void* workspace
   ctx->row_capacity = row_capacity_of(*cfg);
   ctx->elem_bytes = cfg->dtype == UNIPOOL_BF16 ? 2 : 4;
   ctx->tmap_cache = nullptr;
+  ctx->prepared_base = nullptr;
+  ctx->prepared_layers = ctx->prepared_experts = 0;
   cudaError_t e = cudaGetDevice(&ctx->device);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device);
   // the self-cleaning accumulators and the status word start at zero
@@ -220,6 +223,16 @@ int unipool_route(unipool_ctx* ctx, const void* x, int32_t T, const float* W_r, 
   CHECK_PTR(score_sum); CHECK_PTR(znorm); CHECK_PTR(z_saved);
   return route_launch(ctx, x, T, W_r, sigma, bias, n_experts, idx, gate, counts, score_sum,
                       znorm, z_saved, static_cast<cudaStream_t>(stream));
+}
+
+int unipool_router_prepare(unipool_ctx* ctx, const float* W_r, int32_t n_layers, int32_t n_experts,
+                           unipool_stream stream) {
+  CHECK_CTX(ctx);
+  UP_REQUIRE(n_layers >= 0 && n_layers <= ctx->cfg.n_layers, UNIPOOL_ERR_INVALID_ARG,
+             "n_layers = %d outside [0, %d]", n_layers, ctx->cfg.n_layers);
+  if (n_layers > 0) { CHECK_PTR(W_r); CHECK_ROUTER_WIDTH(ctx, n_experts); }
+  if (!use_tensor_cores(ctx)) return UNIPOOL_OK;            // the fp32 path reads W_r itself
+  return router_prepare_launch(ctx, W_r, n_layers, n_experts, static_cast<cudaStream_t>(stream));
 }
 
 int unipool_dispatch(unipool_ctx* ctx, const void* x, int32_t T, const int32_t* idx,

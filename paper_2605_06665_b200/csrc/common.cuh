@@ -53,10 +53,11 @@ struct Workspace {
   double*  dsigma_acc;    // [2]   self-cleaning accumulator of route_bwd / calibrate_c
   int32_t* block_hist;    // [dispatch_blocks, MAX_EXPERTS]
   float*   dz;            // route_bwd scratch: fp32 [max_tokens, pool_size], or bf16 [max_tokens, ceil64(pool_size)]
-  int32_t* split_any;     // [4]   which bf16 terms of the split router weights are non-zero
-  void*    w_split;       // [3, pool_size, d] bf16 terms of the router weights (bf16 mode)
-  int32_t* part_counts;   // [ceil(max_tokens/128), pool_size] per-tile routing counts (bf16 mode)
-  float*   part_sums;     // [ceil(max_tokens/128), pool_size] per-tile score sums
+  int32_t* split_any;     // [n_layers + 1][4] which bf16 terms of a router's split weights are non-zero
+  void*    w_split;       // [n_layers + 1][3, pool_size, d] bf16 terms of the router weights (bf16 mode): one slot
+                          // per prepared layer, the last one scratch for routers that were not prepared
+  int32_t* part_counts;   // [2 ceil(max_tokens/256), pool_size] per-CTA routing counts (bf16 mode)
+  float*   part_sums;     // [2 ceil(max_tokens/256), pool_size] per-CTA score sums
   float*   part_dsigma;   // [ceil(max_tokens/64)] per-block dsigma terms
   void*    dXp;           // [row_capacity, d] expert_bwd scratch (ctx dtype)
   size_t   bytes;         // total
@@ -92,6 +93,8 @@ struct unipool_ctx {
   int64_t row_capacity;
   size_t elem_bytes;
   void* tmap_cache;   // opaque, owned by the tensor-core GEMM module
+  const float* prepared_base;   // router weights last given to unipool_router_prepare (NULL: none)
+  int prepared_layers, prepared_experts;
 };
 
 namespace unipool {
@@ -175,6 +178,7 @@ struct PoolWgradArgs {
 int route_tc_launch(unipool_ctx*, const void* x, int T, const float* W_r, float sigma, const float* bias,
                     int n_experts, int32_t* idx, float* gate, int32_t* counts, float* score_sum,
                     float* znorm, float* z_saved, cudaStream_t);
+int router_prepare_launch(unipool_ctx*, const float* W_r, int n_layers, int n_experts, cudaStream_t);
 int route_bwd_tc_launch(unipool_ctx*, const void* x, int T, const float* W_r, float sigma, int n_experts,
                         const float* znorm, const float* z_saved, const int32_t* idx, const float* dgate,
                         const float* coef, void* dx, float* dW_r, float* dsigma, cudaStream_t);

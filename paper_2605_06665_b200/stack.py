@@ -110,6 +110,7 @@ class UniPoolStack:
             self.sigma[l] = float(r["sigma"])
         if routers[0].get("bias") is not None:
             self.bias = torch.from_numpy(np.stack([r["bias"] for r in routers])).to(self.device)
+        self.ctx.router_prepare(None, 0, self.m)           # forget router terms formed from older weights
         torch.cuda.synchronize(self.device)
 
     def base(self, l):
@@ -148,6 +149,9 @@ class UniPoolStack:
         T = self.T if T is None else T
         if x0 is not None:
             self.x[0, :T].copy_(x0, non_blocking=True)
+        # the routers' weights may have changed since the last pass: one kernel re-forms the bf16 terms
+        # of all layers (used by this forward pass and by the backward pass that follows it)
+        self.ctx.router_prepare(self.W_r, self.L, self.m)
         for l in range(self.L):
             self.forward_layer(l, T)
         return self.x[self.L]
