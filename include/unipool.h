@@ -8,9 +8,11 @@
  * the same calls with a pool view (expert_base, n_experts) per layer.
  *
  * Conventions (all calls)
- *   - Return value: 0 on success, a negative UNIPOOL_ERR_* code otherwise; a
- *     failed call launches nothing.  unipool_last_error() gives the message of
- *     the calling thread's last failure.
+ *   - Return value: 0 on success, a negative UNIPOOL_ERR_* code otherwise.
+ *     Arguments are checked on the host before anything is launched; a CUDA
+ *     or driver error met later in a call that issues several kernels leaves
+ *     the earlier ones queued.  unipool_last_error() gives the message of the
+ *     calling thread's last failure.
  *   - Every tensor pointer is a DEVICE pointer owned by the caller; the library
  *     never allocates or frees device memory.  Scratch lives in the workspace
  *     the caller hands to unipool_create().
@@ -173,7 +175,10 @@ int unipool_dispatch(unipool_ctx* ctx, const void* x, int32_t T, const int32_t* 
  *     rewrite every entry they read, so nothing needs clearing.  Two calls that overlap on the
  *     GPU (different streams) race on it: serialise them.
  *   - An expert index outside [0, n_experts) is dropped (its row_of entry is -1); without a
- *     context there is no status word to report it through. */
+ *     context there is no status word to report it through.
+ *   - Host threads may call concurrently (the per-device look-up is published atomically), but each
+ *     call must be made with the device current whose memory the pointers and `stream` belong to:
+ *     the array's address is looked up for the CURRENT device. */
 int unipool_dispatch_static(const void* x, int32_t T, int32_t d_model, int32_t dtype, int32_t top_k,
                             const int32_t* idx, int32_t n_experts, int64_t row_capacity,
                             int32_t* offsets, int32_t* row_of, int32_t* token_of,
@@ -284,6 +289,14 @@ int unipool_unique_experts(unipool_ctx* ctx, const int32_t* idx, const int32_t* 
  * `stream`, writes the estimate to the HOST float *c_out. */
 int unipool_calibrate_c(unipool_ctx* ctx, int32_t n_experts, int32_t top_k, int32_t n_samples,
                         uint64_t seed, float* c_out, unipool_stream stream);
+
+/* Self-test of the bounded device-side waits (a diagnostic; the paper has no counterpart).  Every
+ * pipeline of the library waits on its barriers for a bounded time and reports an expired wait through
+ * the status word instead of hanging.  This call launches one thread that waits, for at most
+ * limit_cycles SM cycles (0 .. 2e9), on a barrier nobody arrives on: the wait gives up, the kernel
+ * returns normally, and the next unipool_check_status returns UNIPOOL_ERR_TIMEOUT and clears the word.
+ * The context stays usable. */
+int unipool_selftest_wait(unipool_ctx* ctx, int64_t limit_cycles, unipool_stream stream);
 
 /* Per-phase device timing (a measurement aid; the paper has no counterpart).
  * While enabled, every call brackets each of its kernel phases with CUDA events

@@ -25,7 +25,7 @@ EXPORTS = (
     "unipool_expert_fwd", "unipool_combine", "unipool_expert_bwd", "unipool_pool_wgrad",
     "unipool_pool_aux_loss", "unipool_route_bwd", "unipool_calibrate_c",
     "unipool_profile_enable", "unipool_profile_read", "unipool_dispatch_static",
-    "unipool_unique_experts", "unipool_router_prepare",
+    "unipool_unique_experts", "unipool_router_prepare", "unipool_selftest_wait",
 )
 
 PHASES = (
@@ -102,6 +102,8 @@ def lib():
     L.unipool_unique_experts.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp]
     L.unipool_calibrate_c.restype = ctypes.c_int
     L.unipool_calibrate_c.argtypes = [vp, i32, i32, i32, ctypes.c_uint64, ctypes.POINTER(f32), vp]
+    L.unipool_selftest_wait.restype = ctypes.c_int
+    L.unipool_selftest_wait.argtypes = [vp, i64, vp]
     L.unipool_profile_enable.restype = ctypes.c_int
     L.unipool_profile_enable.argtypes = [vp, i32]
     L.unipool_profile_read.restype = ctypes.c_int
@@ -181,6 +183,9 @@ class Context:
     def route(self, x, T, W_r, sigma, bias, n_experts, idx, gate, counts, score_sum, znorm, z_saved):
         _check(lib().unipool_route(self.handle, _p(x), T, _p(W_r), sigma, _p(bias), n_experts, _p(idx),
                                    _p(gate), _p(counts), _p(score_sum), _p(znorm), _p(z_saved), _stream()))
+
+    def selftest_wait(self, limit_cycles):
+        _check(lib().unipool_selftest_wait(self.handle, int(limit_cycles), _stream()))
 
     def router_prepare(self, W_r, n_layers, n_experts):
         _check(lib().unipool_router_prepare(self.handle, _p(W_r), n_layers, n_experts, _stream()))

@@ -19,13 +19,7 @@ void set_error(const char* fmt, ...) {
   va_end(ap);
 }
 
-// Debug aid: UNIPOOL_FORCE_SIMT=1 runs the bf16 grouped GEMMs on the CUDA-core path
-// (same arithmetic contract, far slower); used to bisect tensor-core issues.
-bool force_simt() {
-  static const bool forced = [] { const char* v = getenv("UNIPOOL_FORCE_SIMT"); return v && v[0] == '1'; }();
-  return forced;
-}
-static bool use_tensor_cores(const unipool_ctx* ctx) { return ctx->cfg.dtype == UNIPOOL_BF16 && !force_simt(); }
+static bool use_tensor_cores(const unipool_ctx* ctx) { return ctx->cfg.dtype == UNIPOOL_BF16; }
 
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -297,6 +291,9 @@ int unipool_pool_wgrad(unipool_ctx* ctx, int32_t n_layers, int64_t layer_stride_
   UP_REQUIRE(n_layers >= 1, UNIPOOL_ERR_INVALID_ARG, "n_layers must be >= 1");
   UP_REQUIRE(layer_stride_rows >= 0 && layer_stride_rows % UNIPOOL_ROW_ALIGN == 0,
              UNIPOOL_ERR_INVALID_ARG, "layer_stride_rows must be a multiple of %d", UNIPOOL_ROW_ALIGN);
+  UP_REQUIRE((int64_t)n_layers * layer_stride_rows < (1ll << 31) && (n_layers == 1 || layer_stride_rows > 0),
+             UNIPOOL_ERR_UNSUPPORTED, "n_layers * layer_stride_rows = %lld must stay below 2^31 rows",
+             (long long)n_layers * (long long)layer_stride_rows);
   CHECK_PTR(offsets);
   UP_REQUIRE(dW_gu != nullptr || dW_down != nullptr, UNIPOOL_ERR_INVALID_ARG, "dW_gu and dW_down are both NULL");
   if (dW_gu != nullptr) { CHECK_PTR(Xp); CHECK_PTR(dGU); }
@@ -338,6 +335,13 @@ int unipool_unique_experts(unipool_ctx* ctx, const int32_t* idx, const int32_t* 
   UP_REQUIRE(L >= 1, UNIPOOL_ERR_INVALID_ARG, "L must be >= 1");
   return unique_experts_launch(ctx, idx, expert_base, L, T, unique, reinterpret_cast<unsigned long long*>(total),
                                static_cast<cudaStream_t>(stream));
+}
+
+int unipool_selftest_wait(unipool_ctx* ctx, int64_t limit_cycles, unipool_stream stream) {
+  CHECK_CTX(ctx);
+  UP_REQUIRE(limit_cycles >= 0 && limit_cycles <= 2000000000ll, UNIPOOL_ERR_INVALID_ARG,
+             "limit_cycles = %lld outside [0, 2e9]", (long long)limit_cycles);
+  return wait_selftest_launch(ctx, limit_cycles, static_cast<cudaStream_t>(stream));
 }
 
 int unipool_calibrate_c(unipool_ctx* ctx, int32_t n_experts, int32_t top_k, int32_t n_samples,

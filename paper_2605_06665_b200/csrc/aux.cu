@@ -1,5 +1,6 @@
 // Pool-level balance loss (Eqs. 4-5) and the Monte-Carlo constant c (Alg. 1).
 #include "common.cuh"
+#include "tc_ptx.cuh"
 
 namespace unipool {
 
@@ -149,6 +150,32 @@ int calibrate_launch(unipool_ctx* ctx, int E, int k, int n_samples, uint64_t see
   UP_CUDA(cudaStreamSynchronize(s));
   UP_REQUIRE(host[1] > 0.0, UNIPOOL_ERR_DEVICE_CHECK, "calibrate_c: no usable sample");
   *c_out = (float)(host[0] / host[1]);
+  return UNIPOOL_OK;
+}
+
+// Exercises the bounded wait every pipeline of the library is built on: one thread waits, for at most
+// limit_cycles SM cycles, on an mbarrier that nobody arrives on.  The wait gives up, the kernel records
+// the time-out in the status word the way the GEMM and router kernels do, and returns normally.
+__global__ void wait_selftest_kernel(long long limit_cycles, int32_t* status) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    tc::mbar_init(&bar, 1);
+    tc::fence_barrier_init();
+    if (!tc::mbar_wait(&bar, 0, &abort_flag, limit_cycles)) {
+      abort_flag = 1;
+      if (atomicCAS(status, 0, kStatusTimeout) == 0) {
+        status[1] = 99;                                   // site code of this self-test
+        status[2] = 0;
+      }
+    }
+  }
+}
+
+int wait_selftest_launch(unipool_ctx* ctx, long long limit_cycles, cudaStream_t s) {
+  wait_selftest_kernel<<<1, 32, 0, s>>>(limit_cycles, ctx->ws.status);
+  UP_LAUNCH_CHECK();
   return UNIPOOL_OK;
 }
 

@@ -13,7 +13,6 @@ namespace unipool {
 
 // ---------------------------------------------------------------- errors
 void set_error(const char* fmt, ...);
-bool force_simt();   // debug aid: UNIPOOL_FORCE_SIMT=1 runs the bf16 mode on the CUDA-core kernels
 
 #define UP_REQUIRE(cond, code, ...)      \
   do {                                   \
@@ -155,6 +154,7 @@ int aux_launch(unipool_ctx*, const int32_t* counts, const float* S, int L, int n
                cudaStream_t);
 int unique_experts_launch(unipool_ctx*, const int32_t* idx, const int32_t* expert_base, int L, int T,
                           int32_t* unique, unsigned long long* total, cudaStream_t);
+int wait_selftest_launch(unipool_ctx*, long long limit_cycles, cudaStream_t);
 int calibrate_launch(unipool_ctx*, int n_experts, int top_k, int n_samples, uint64_t seed,
                      float* c_out, cudaStream_t);
 

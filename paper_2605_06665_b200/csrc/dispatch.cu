@@ -1,5 +1,7 @@
 // Token permute into expert-contiguous order and its inverse (combine), forward
 // and backward.  All data movement is in 16-byte vectors; one warp moves one row.
+#include <atomic>
+
 #include "common.cuh"
 
 namespace unipool {
@@ -453,8 +455,12 @@ namespace {
 constexpr int64_t kStaticHistInts = 1024 * 512 - 64;      // chunks x experts that fit
 static __device__ __align__(256) int32_t g_dispatch_scratch[1024 * 512];
 constexpr int kMaxDevices = 64;
-int32_t* g_scratch_addr[kMaxDevices] = {};
-int g_scratch_sms[kMaxDevices] = {};
+// per device: the array's address there and the SM count, looked up by the first call on that device.
+// Host threads may race on the first call: the entry is complete before its address becomes visible.
+struct ScratchInfo { int32_t* addr; int sms; };
+std::atomic<const ScratchInfo*> g_scratch[kMaxDevices];
+ScratchInfo g_scratch_slots[kMaxDevices][2];
+std::atomic<int> g_scratch_next[kMaxDevices];
 }  // namespace
 
 extern "C" int unipool_dispatch_static(const void* x, int32_t T, int32_t d_model, int32_t dtype, int32_t top_k,
@@ -486,18 +492,23 @@ extern "C" int unipool_dispatch_static(const void* x, int32_t T, int32_t d_model
   UP_CUDA(cudaGetDevice(&dev));
   UP_REQUIRE(dev >= 0 && dev < kMaxDevices, UNIPOOL_ERR_UNSUPPORTED, "dispatch_static: device ordinal %d", dev);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (g_scratch_addr[dev] == nullptr) {
+  const ScratchInfo* info = g_scratch[dev].load(std::memory_order_acquire);
+  if (info == nullptr) {
     // Once per device, with that device current: in host code the array's name is only a handle,
-    // the kernels need the address it has on THIS device.
+    // the kernels need the address it has on THIS device.  Two threads that both get here look up the
+    // same values; each fills a slot of its own and publishes it.
     int32_t* ptr = nullptr;
     UP_CUDA(cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_dispatch_scratch));
     int sms = 0;
     UP_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    g_scratch_sms[dev] = sms;
-    g_scratch_addr[dev] = ptr;
+    UP_REQUIRE(ptr != nullptr && sms > 0, UNIPOOL_ERR_CUDA, "dispatch_static: no address for the built-in scratch");
+    const int slot = g_scratch_next[dev].fetch_add(1) & 1;
+    g_scratch_slots[dev][slot] = ScratchInfo{ptr, sms};
+    g_scratch[dev].store(&g_scratch_slots[dev][slot], std::memory_order_release);
+    info = &g_scratch_slots[dev][slot];
   }
-  int32_t* status = g_scratch_addr[dev];                   // [0, 64): status word (+ spare)
-  int32_t* bh = g_scratch_addr[dev] + 64;                  // per-chunk histograms / bases
+  int32_t* status = info->addr;                            // [0, 64): status word (+ spare)
+  int32_t* bh = info->addr + 64;                           // per-chunk histograms / bases
   const int cap = (int)row_capacity;
   if (T == 0) {
     dispatch_empty_kernel<<<(cap + 255) / 256, 256, 0, s>>>(offsets, token_of, tile_expert, n_experts, cap);
@@ -513,7 +524,7 @@ extern "C" int unipool_dispatch_static(const void* x, int32_t T, int32_t d_model
   dispatch_rank_kernel<<<n_blocks, kDispatchWarps * 32, kDispatchWarps * n_experts * sizeof(int), s>>>(idx, T, top_k, n_experts, bh, row_of, token_of);
   UP_LAUNCH_CHECK();
   const int row_vecs = (int)((size_t)d_model * eb / 16);
-  int64_t want = ((int64_t)cap + 7) / 8, lim = (int64_t)g_scratch_sms[dev] * 8;
+  int64_t want = ((int64_t)cap + 7) / 8, lim = (int64_t)info->sms * 8;
   const int grid = (int)(want < 1 ? 1 : (want < lim ? want : lim));
   gather_rows_kernel<<<grid, 256, 0, s>>>(static_cast<const uint4*>(x), token_of, offsets + n_experts,
                                           static_cast<uint4*>(Xp), row_vecs, cap);

@@ -17,8 +17,6 @@
 //                                 for a group's odd last tile)
 #include <cuda.h>
 
-#include <cstdlib>
-
 #include "common.cuh"
 #include "tc_ptx.cuh"
 
@@ -56,8 +54,6 @@ struct GemmParams {
   const int32_t* offsets;       // row tiles: &offsets[n_experts]; wgrad: [n_layers][n_experts+1]
   const int32_t* tile_expert;   // row tiles only
   const int32_t* group_offsets; // row tiles on CTA pairs: [n_experts + 1] starts of the groups
-  int part;                     // row tiles: 0 = every tile; 1 = pair kernel, whole pairs only (a group's odd last
-                                // tile is left out); 2 = single-CTA kernel, only those odd last tiles
   int n_experts, expert_base;
   int n_layers;                 // wgrad
   int layer_stride_rows;        // wgrad
@@ -84,13 +80,10 @@ template <int MODE> struct Traits {
 
 struct TileCoord { int e, mt, nt, kblocks; bool valid; int col0, ncols; };   // output columns [col0, col0 + ncols)
 
-// `odd` (row tiles with p.part == 2): odd[e] = groups before expert e that have an odd number of row
-// tiles; the kernel then visits only the last tile of those groups.
 template <int MODE>
-__device__ __forceinline__ int tiles_total(const GemmParams& p, int& n_nt, int& n_mt, const uint16_t* odd) {
+__device__ __forceinline__ int tiles_total(const GemmParams& p, int& n_nt, int& n_mt) {
   if constexpr (Traits<MODE>::kRowTiles) {
     n_mt = p.offsets ? *p.offsets / BM : p.Mdim;     // no offsets: one group of Mdim row tiles
-    if (p.part == 2) n_mt = odd[p.n_experts];
     const int ncols = MODE == kFwd1 ? BN / 2 : BN;
     n_nt = (p.Ndim + ncols - 1) / ncols;
     return n_mt * n_nt;
@@ -102,26 +95,9 @@ __device__ __forceinline__ int tiles_total(const GemmParams& p, int& n_nt, int& 
 }
 
 template <int MODE>
-__device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int tile, int n_nt, int n_mt,
-                                                const uint16_t* odd = nullptr) {
+__device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int tile, int n_nt, int n_mt) {
   TileCoord c;
   if constexpr (Traits<MODE>::kRowTiles) {
-    if (p.part == 2) {                               // the j-th odd group's last tile
-      const int j = tile / n_nt;
-      int lo = 0, hi = p.n_experts - 1;              // last e with odd[e] <= j: the group itself is odd
-      while (lo < hi) {
-        const int mid = (lo + hi + 1) >> 1;
-        if ((int)odd[mid] <= j) lo = mid; else hi = mid - 1;
-      }
-      c.e = lo;
-      c.mt = p.group_offsets[lo + 1] / BM - 1;
-      c.nt = tile % n_nt;
-      c.kblocks = p.Kdim / BK;
-      c.valid = true;
-      c.col0 = c.nt * BN;
-      c.ncols = BN;
-      return c;
-    }
     // A kernel that consumes what the previous launch produced in ascending row order (the down
     // projection reads A, the second dgrad reads dGU) walks the rows downwards: the rows written
     // last are the ones still in L2.
@@ -168,7 +144,7 @@ __device__ __forceinline__ TailSplit tail_split(const GemmParams& p, int total) 
   if constexpr (MODE == kFwd2 || MODE == kDgrad2) {
     const int grid = (int)gridDim.x;
     const int rest = total % grid;
-    if (p.part == 0 && rest > 0 && 2 * rest <= grid) {
+    if (rest > 0 && 2 * rest <= grid) {
       t.full = total - rest;
       t.slices = 4 * rest <= grid ? 4 : 2;
       t.units = t.full + rest * t.slices;
@@ -177,11 +153,10 @@ __device__ __forceinline__ TailSplit tail_split(const GemmParams& p, int total) 
   return t;
 }
 template <int MODE>
-__device__ __forceinline__ TileCoord unit_coord(const GemmParams& p, const TailSplit& ts, int unit, int n_nt, int n_mt,
-                                                const uint16_t* odd) {
-  if (unit < ts.full) return tile_coord<MODE>(p, unit, n_nt, n_mt, odd);
+__device__ __forceinline__ TileCoord unit_coord(const GemmParams& p, const TailSplit& ts, int unit, int n_nt, int n_mt) {
+  if (unit < ts.full) return tile_coord<MODE>(p, unit, n_nt, n_mt);
   const int u = unit - ts.full;
-  TileCoord c = tile_coord<MODE>(p, ts.full + u / ts.slices, n_nt, n_mt, odd);
+  TileCoord c = tile_coord<MODE>(p, ts.full + u / ts.slices, n_nt, n_mt);
   c.ncols = BN / ts.slices;
   c.col0 += (u % ts.slices) * c.ncols;
   return c;
@@ -377,19 +352,8 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
   tc::tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_ptr;
 
-  uint16_t* odd = reinterpret_cast<uint16_t*>(smem + kBarOffset + 512);     // [n_experts + 1], row tiles with part == 2
-  if constexpr (TR::kRowTiles) {
-    if (p.part == 2) {
-      for (int e = threadIdx.x; e <= p.n_experts; e += blockDim.x) {
-        int before = 0;
-        for (int o = 0; o < e; ++o) before += ((p.group_offsets[o + 1] - p.group_offsets[o]) / BM) & 1;
-        odd[e] = (uint16_t)before;
-      }
-      __syncthreads();
-    }
-  }
   int n_nt, n_mt;
-  const int n_tiles = tiles_total<MODE>(p, n_nt, n_mt, odd);
+  const int n_tiles = tiles_total<MODE>(p, n_nt, n_mt);
   const TailSplit ts = tail_split<MODE>(p, n_tiles);
   const int total = ts.units;                        // work units: whole tiles, then slices of the last round
 
@@ -400,7 +364,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
       uint32_t phase = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
-        const TileCoord c = unit_coord<MODE>(p, ts, tile, n_nt, n_mt, odd);
+        const TileCoord c = unit_coord<MODE>(p, ts, tile, n_nt, n_mt);
         if (!c.valid) continue;
         const int pe = p.expert_base + c.e;
         int layer = 0, r = 0, r_end = 0;              // wgrad: walks the rows of expert e, layer by layer
@@ -471,7 +435,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
       int local = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
-        const TileCoord c = unit_coord<MODE>(p, ts, tile, n_nt, n_mt, odd);
+        const TileCoord c = unit_coord<MODE>(p, ts, tile, n_nt, n_mt);
         if (!c.valid) continue;
         const int acc = local & 1;
         const uint32_t acc_phase = (local >> 1) & 1;
@@ -558,7 +522,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     int local = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
-      const TileCoord c = unit_coord<MODE>(p, ts, tile, n_nt, n_mt, odd);
+      const TileCoord c = unit_coord<MODE>(p, ts, tile, n_nt, n_mt);
       if (!c.valid) {
         if constexpr (MODE == kWgrad) {
           if (p.overwrite) {                           // no rows anywhere: the gradient of this tile is zero
@@ -1053,11 +1017,10 @@ row_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     tc::tmem_relinquish_pair();
   }
   // pair-tiles before each expert: an expert of n row tiles takes ceil(n / 2), the last one a half
-  // pair-tile when n is odd (part 1: floor(n / 2), the odd last tile is another kernel's)
+  // pair-tile when n is odd
   for (int e = threadIdx.x; e <= p.n_experts; e += blockDim.x) {
     int before = 0;
-    const int round_up = p.part == 1 ? 0 : 1;
-    for (int o = 0; o < e; ++o) before += ((p.group_offsets[o + 1] - p.group_offsets[o]) / BM + round_up) >> 1;
+    for (int o = 0; o < e; ++o) before += ((p.group_offsets[o + 1] - p.group_offsets[o]) / BM + 1) >> 1;
     pp[e] = (uint16_t)before;
   }
   tc::tc_fence_before_sync();
@@ -1212,55 +1175,42 @@ int launch(unipool_ctx* ctx, int phase, const CUtensorMap& tmA, const CUtensorMa
   return UNIPOOL_OK;
 }
 
-// How the row-tile GEMMs (gate/up, down, second dgrad) of a call are scheduled:
-//   kRowsSingle  every tile on the single-CTA kernel;
-//   kRowsPairs   every tile on CTA pairs (the odd last tile of a group as a half pair-tile, M = 128);
-//   kRowsSplit   whole pairs on the pair kernel, then the odd last tiles on the single-CTA kernel.
-// Pairs move a third fewer operand bytes into the SMs.  Measured (interleaved runs, one B200), pairs
-// against single per GEMM: -10 % at 32 row tiles per group, -3 .. -8 % at 4 - 7 tiles, none at 2.7
-// tiles (341 rows), where two thirds of the operand bytes miss L2 and each k-block waits for the slower
-// of two CTAs' loads.  The split schedule streams every weight twice (once per kernel) and is 19 %
-// slower than single at 2.7 tiles.  So: pairs when a batch of max_tokens gives the average expert four
-// row tiles, single otherwise; UNIPOOL_ROW_PAIR = 0 / 1 / 2 forces single / pairs / split (a
-// debugging aid).  The pair schedule keeps 16-bit counts of pair-tiles.
-enum RowPlan { kRowsSingle = 0, kRowsPairs = 1, kRowsSplit = 2 };
-RowPlan row_plan(const unipool_ctx* ctx, int n_experts) {
-  static const int forced = [] { const char* v = getenv("UNIPOOL_ROW_PAIR"); return v ? v[0] - '0' : -1; }();
-  if (ctx->sm_count < 2 || ctx->row_capacity / (2 * BM) + n_experts >= 65535) return kRowsSingle;
-  if (forced >= 0 && forced <= 2) return static_cast<RowPlan>(forced);
-  return (int64_t)ctx->cfg.max_tokens * ctx->cfg.top_k >= (int64_t)4 * BM * n_experts ? kRowsPairs : kRowsSingle;
+// The row-tile GEMMs (gate/up, down, second dgrad) of a call run either all on the single-CTA kernel or
+// all on CTA pairs (the odd last tile of a group as a half pair-tile, M = 128).  Pairs move a third
+// fewer operand bytes into the SMs.  Measured (interleaved runs, one B200), pairs against single per
+// GEMM: -10 % at 32 row tiles per group, -3 .. -8 % at 4 - 7 tiles, none at 2.7 tiles (341 rows): a
+// half pair-tile uses the tensor cores at half rate, and every third tile is one.  So: pairs when a
+// batch of max_tokens gives the average expert four row tiles, single otherwise.  The pair schedule
+// keeps 16-bit counts of pair-tiles.
+bool rows_on_pairs(const unipool_ctx* ctx, int n_experts) {
+  if (ctx->sm_count < 2 || ctx->row_capacity / (2 * BM) + n_experts >= 65535) return false;
+  return (int64_t)ctx->cfg.max_tokens * ctx->cfg.top_k >= (int64_t)4 * BM * n_experts;
 }
 
-// One row-tile GEMM under `plan`.  tmA / tmB: the operand maps of the single-CTA kernel; tmA64 / tmBp:
-// those of the pair kernel's half pair-tiles (64-row boxes of A) and of its B halves (64-row boxes).
+// One row-tile GEMM.  tmA / tmB: the operand maps of the single-CTA kernel; tmA64 / tmBp: those of the
+// pair kernel's half pair-tiles (64-row boxes of A) and of its B halves (64-row boxes).
 template <int MODE>
-int launch_rows(unipool_ctx* ctx, int phase, RowPlan plan, const CUtensorMap& tmA, const CUtensorMap& tmA64,
+int launch_rows(unipool_ctx* ctx, int phase, bool pairs, const CUtensorMap& tmA, const CUtensorMap& tmA64,
                 const CUtensorMap& tmB, const CUtensorMap& tmBp, const CUtensorMap& tmC0, const CUtensorMap& tmC1,
-                GemmParams p, cudaStream_t s) {
-  PhaseTimer pt(ctx, phase, plan == kRowsSplit ? 2 : 1, s);
-  if (plan != kRowsSingle) {
-    p.part = plan == kRowsSplit ? 1 : 0;
+                const GemmParams& p, cudaStream_t s) {
+  PhaseTimer pt(ctx, phase, 1, s);
+  if (pairs) {
     auto kern = row_pair_kernel<MODE>;
     UP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPairSmemTotal));
     kern<<<ctx->sm_count / 2 * 2, kRowPairThreads, kPairSmemTotal, s>>>(tmA, tmA64, tmBp, tmC0, tmC1, p);
-    UP_LAUNCH_CHECK();
-  }
-  if (plan != kRowsPairs) {
-    p.part = plan == kRowsSplit ? 2 : 0;
+  } else {
     auto kern = grouped_gemm_tc_kernel<MODE>;
     UP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemTotal));
     kern<<<ctx->sm_count, Traits<MODE>::kThreads, kSmemTotal, s>>>(tmA, tmB, tmC0, tmC1, p);
-    UP_LAUNCH_CHECK();
   }
+  UP_LAUNCH_CHECK();
   return UNIPOOL_OK;
 }
 
-// The pool weight gradient runs on CTA pairs (UNIPOOL_WGRAD_PAIR=0, a debugging aid, selects the
-// single-CTA kernel).
+// The pool weight gradient runs on CTA pairs (a device with a single SM falls back to the single-CTA kernel).
 int launch_wgrad(unipool_ctx* ctx, int phase, const CUtensorMap& tmP, const CUtensorMap& tmQ, const CUtensorMap& tmW,
                  const GemmParams& p, cudaStream_t s) {
-  static const bool pair = [] { const char* v = getenv("UNIPOOL_WGRAD_PAIR"); return !(v && v[0] == '0'); }();
-  if (!pair || ctx->sm_count < 2) return launch<kWgrad>(ctx, phase, tmP, tmQ, tmW, tmW, p, s);
+  if (ctx->sm_count < 2) return launch<kWgrad>(ctx, phase, tmP, tmQ, tmW, tmW, p, s);
   PhaseTimer pt(ctx, phase, 1, s);
   UP_CUDA(cudaFuncSetAttribute(wgrad_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPairSmemTotal));
   wgrad_pair_kernel<<<ctx->sm_count / 2 * 2, kThreads, kPairSmemTotal, s>>>(tmP, tmQ, tmW, p);
@@ -1326,7 +1276,7 @@ int expert_fwd_tc(unipool_ctx* ctx, const ExpertFwdArgs& a, cudaStream_t s) {
   p.f = f;
   p.status = ctx->ws.status;
   p.group_offsets = a.offsets;
-  const RowPlan plan = row_plan(ctx, a.n_experts);
+  const bool plan = rows_on_pairs(ctx, a.n_experts);
   CUtensorMap tmA, tmA64, tmB, tmBp, tmC0, tmC1;
   int rc;
   // GU = Xp [W_gate; W_up]^T with the SwiGLU epilogue.  B tile = 128 gate rows + 128 up rows of the
@@ -1384,7 +1334,7 @@ int expert_bwd_tc(unipool_ctx* ctx, const ExpertBwdArgs& a, cudaStream_t s) {
   p.group_offsets = a.offsets;
   CUtensorMap tmA64;
   if ((rc = map_2d(ctx, &tmA64, a.dGU, 2 * f, cap, 64, 64)) != UNIPOOL_OK) return rc;
-  rc = launch_rows<kDgrad2>(ctx, UNIPOOL_PH_DGRAD_GU, row_plan(ctx, a.n_experts), tmA, tmA64, tmB, tmB, tmC0, tmC0, p, s);
+  rc = launch_rows<kDgrad2>(ctx, UNIPOOL_PH_DGRAD_GU, rows_on_pairs(ctx, a.n_experts), tmA, tmA64, tmB, tmB, tmC0, tmC0, p, s);
   if (rc != UNIPOOL_OK) return rc;
   if (a.wgrad) {
     PoolWgradArgs w{1, 0, a.offsets, a.Xp, a.A, a.dYp, a.dGU, a.expert_base, a.n_experts, a.dW_gu, a.dW_down,

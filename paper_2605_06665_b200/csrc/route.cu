@@ -162,7 +162,7 @@ int route_launch(unipool_ctx* ctx, const void* x, int T, const float* W_r, float
     UP_LAUNCH_CHECK();
     return UNIPOOL_OK;
   }
-  if (ctx->cfg.dtype == UNIPOOL_BF16 && !force_simt())
+  if (ctx->cfg.dtype == UNIPOOL_BF16)
     return route_tc_launch(ctx, x, T, W_r, sigma, bias, M, idx, gate, counts, score_sum, znorm, z_saved, s);
   dim3 g1((T + kSimtTile - 1) / kSimtTile, (M + kSimtTile - 1) / kSimtTile);
   {
@@ -312,7 +312,7 @@ int route_bwd_launch(unipool_ctx* ctx, const void* x, int T, const float* W_r, f
                      const float* dgate, const float* coef, void* dx, float* dW_r, float* dsigma,
                      cudaStream_t s) {
   if (T == 0) return UNIPOOL_OK;
-  if (ctx->cfg.dtype == UNIPOOL_BF16 && !force_simt())
+  if (ctx->cfg.dtype == UNIPOOL_BF16)
     return route_bwd_tc_launch(ctx, x, T, W_r, sigma, M, znorm, z_saved, idx, dgate, coef, dx, dW_r, dsigma, s);
   const int d = ctx->cfg.d_model, k = ctx->cfg.top_k;
   float* dz = ctx->ws.dz;

@@ -42,14 +42,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // ~kWaitCycles SM cycles or as soon as another role has raised *abort; returns
 // false in both cases (the caller leaves its loop).
 constexpr long long kWaitCycles = 4000000000ll;   // about two seconds
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort,
+                                          long long limit_cycles = kWaitCycles) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (uint32_t it = 1;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 255u) == 0u) {
       if (*abort) return false;
-      if (clock64() - t0 > kWaitCycles) return false;
+      if (clock64() - t0 > limit_cycles) return false;
     }
   }
 }

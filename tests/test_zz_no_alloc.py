@@ -68,3 +68,48 @@ def test_dispatch_static_refuses_what_does_not_fit():
     with pytest.raises(B.UniPoolError) as ei:
         B.dispatch_static(one, T, d, B.FP32, k, one, M, cap, one, one, one, one, one)
     assert ei.value.code == -3 and "scratch" in str(ei.value)
+
+
+def test_dispatch_static_without_tokens_and_with_a_bad_index():
+    """Two corners of the entry point: T = 0 leaves empty maps, and an expert id outside the router's
+    range is dropped (row_of = -1; there is no status word to report it through) while every other
+    assignment keeps the row the reference call gives it."""
+    import torch
+    from paper_2605_06665_b200 import binding as B
+    d, f, k, M = 128, 128, 2, 16
+    T = 700
+    cfg = B.make_config(d, f, M, k, 1, T, B.FP32, 1e-6, 2.0)
+    ctx = B.Context(cfg, "cuda")
+    cap = ctx.row_capacity
+    i32 = torch.int32
+    g = torch.Generator(device="cpu").manual_seed(11)
+    x = torch.randn(T, d, generator=g).cuda()
+    idx = torch.rand(T, M, generator=g).topk(k, dim=1).indices.to(i32).cuda()
+
+    def outputs():
+        return dict(offsets=torch.full((M + 1,), -7, dtype=i32, device="cuda"),
+                    row_of=torch.full((T, k), -7, dtype=i32, device="cuda"),
+                    token_of=torch.full((cap,), -7, dtype=i32, device="cuda"),
+                    tile_expert=torch.full((cap // B.ROW_ALIGN,), -7, dtype=i32, device="cuda"),
+                    Xp=torch.zeros(cap, d, device="cuda"))
+
+    o = outputs()
+    B.dispatch_static(x, 0, d, B.FP32, k, idx, M, cap, o["offsets"], o["row_of"], o["token_of"], o["tile_expert"], o["Xp"])
+    torch.cuda.synchronize()
+    assert not o["offsets"].any() and (o["token_of"] == -1).all() and (o["tile_expert"] == -1).all()
+
+    bad = idx.clone()
+    bad[5, 1] = M + 3                                        # out of range: dropped
+    ref, got = outputs(), outputs()
+    ctx.dispatch(x, T, bad, M, ref["offsets"], ref["row_of"], ref["token_of"], ref["tile_expert"], ref["Xp"])
+    B.dispatch_static(x, T, d, B.FP32, k, bad, M, cap, got["offsets"], got["row_of"], got["token_of"],
+                      got["tile_expert"], got["Xp"])
+    torch.cuda.synchronize()
+    with pytest.raises(B.UniPoolError):                      # the context's call reports it ...
+        ctx.check_status()
+    assert int(got["row_of"][5, 1]) == -1                    # ... the static one can only drop it
+    assert torch.equal(got["row_of"], ref["row_of"]) and torch.equal(got["offsets"], ref["offsets"])
+    assert torch.equal(got["token_of"], ref["token_of"])
+    assert int(got["offsets"][M]) >= T * k - 1
+    ctx.close()
+
