@@ -313,6 +313,7 @@ __device__ __forceinline__ void epilogue_rows(const CUtensorMap* tmC0, const Gem
 template <int MODE>
 __global__ void __launch_bounds__(Traits<MODE>::kThreads, 1)
 grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                       const __grid_constant__ CUtensorMap tmB64,   // dgrad: 64 x 64 boxes of the weights (column slices)
                        const __grid_constant__ CUtensorMap tmC0, const __grid_constant__ CUtensorMap tmC1,
                        const GemmParams p) {
   using TR = Traits<MODE>;
@@ -395,11 +396,13 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
             }
           } else if constexpr (MODE == kDgrad1 || MODE == kDgrad2) {
             tc::tma_load_2d(sA, &tmA, &full_bar[stage], kb * BK, c.mt * BM);
-#pragma unroll
-            for (int i = 0; i < BN / 64; ++i)
-              if (64 * i < c.ncols)
-                tc::tma_load_2d(sB + i * kMnBlockBytes, &tmB, &full_bar[stage], c.col0 + 64 * i,
+            if (c.ncols == BN) {                      // the four 64-column blocks of the weights in one box
+              tc::tma_load_3d(sB, &tmB, &full_bar[stage], 0, pe * p.Kdim + kb * BK, c.col0 / 64);
+            } else {
+              for (int i = 0; i < c.ncols / 64; ++i)
+                tc::tma_load_2d(sB + i * kMnBlockBytes, &tmB64, &full_bar[stage], c.col0 + 64 * i,
                                 pe * p.Kdim + kb * BK);
+            }
           } else {
             while (r >= r_end) {                        // next layer that has rows for this expert
               ++layer;
@@ -408,12 +411,8 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
               r_end = off[c.e + 1];
             }
             const int grow = layer * p.layer_stride_rows + r;
-#pragma unroll
-            for (int i = 0; i < BM / 64; ++i)
-              tc::tma_load_2d(sA + i * kMnBlockBytes, &tmA, &full_bar[stage], c.mt * BM + 64 * i, grow);
-#pragma unroll
-            for (int i = 0; i < BN / 64; ++i)
-              tc::tma_load_2d(sB + i * kMnBlockBytes, &tmB, &full_bar[stage], c.nt * BN + 64 * i, grow);
+            tc::tma_load_3d(sA, &tmA, &full_bar[stage], 0, grow, c.mt * (BM / 64));   // two 64-column blocks
+            tc::tma_load_3d(sB, &tmB, &full_bar[stage], 0, grow, c.nt * (BN / 64));   // four
             r += BK;
           }
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
@@ -754,11 +753,9 @@ wgrad_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           uint8_t* sA = smem + stage * kPairStageBytes;
           uint8_t* sB = sA + kPairHalfBytes;
           if (rank == 0) tc::mbar_expect_tx(&full_bar[stage], 2 * kPairStageBytes);   // both CTAs' bytes
-#pragma unroll
-          for (int i = 0; i < 2; ++i) {
-            tc::tma_load_2d_pair(sA + i * kMnBlockBytes, &tmA, &full_bar[stage], mt * 256 + rank * 128 + 64 * i, grow);
-            tc::tma_load_2d_pair(sB + i * kMnBlockBytes, &tmB, &full_bar[stage], nt * 256 + rank * 128 + 64 * i, grow);
-          }
+          // this CTA's two 64-column blocks of each operand, one box each
+          tc::tma_load_3d_pair(sA, &tmA, &full_bar[stage], 0, grow, mt * 4 + rank * 2);
+          tc::tma_load_3d_pair(sB, &tmB, &full_bar[stage], 0, grow, nt * 4 + rank * 2);
           r += BK;
           if (++stage == kPairStages) { stage = 0; phase ^= 1u; }
         }
@@ -925,6 +922,16 @@ int map_2d(const unipool_ctx* ctx, CUtensorMap* out, const void* base, uint64_t 
   return make_tmap(ctx, out, kind, base, 2, dims, strides, box);
 }
 
+// MMA operand read along the contiguous dimension of a row-major matrix [k_rows, n_cols] ("MN-major"):
+// the matrix seen as [n_cols / 64][k_rows][64], a box = `blocks` column blocks x 64 k-rows, laid out
+// block after block (8 KiB each) - one copy instead of one per block.
+int map_mn(const unipool_ctx* ctx, CUtensorMap* out, const void* base, uint64_t n_cols, uint64_t k_rows,
+           uint32_t blocks) {
+  const uint64_t dims[3] = {64, k_rows, n_cols / 64}, strides[2] = {n_cols, 64};
+  const uint32_t box[3] = {64, 64, blocks};
+  return make_tmap(ctx, out, kMapOperand, base, 3, dims, strides, box);
+}
+
 // 32 x 32 epilogue chunk map
 int map_chunk(const unipool_ctx* ctx, CUtensorMap* out, const void* base, uint64_t cols, uint64_t rows,
               MapKind kind) {
@@ -1052,20 +1059,12 @@ row_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
           if (rank == 0) tc::mbar_expect_tx(&full_bar[stage], tx);              // both CTAs' bytes
           if (t.half) tc::tma_load_2d_pair(sA, &tmA64, &full_bar[stage], kb * BK, t.mt * BM + rank * (BM / 2));
           else tc::tma_load_2d_pair(sA, &tmA, &full_bar[stage], kb * BK, (t.mt + rank) * BM);
-          if constexpr (MODE == kFwd1) {           // 64 gate features, then the same 64 up features
-            const int feat = t.nt * (BN / 2) + rank * 64;
-            tc::tma_load_2d_pair(sB, &tmB, &full_bar[stage], kb * BK, pe * 2 * p.f + feat);
-            tc::tma_load_2d_pair(sB + kMnBlockBytes, &tmB, &full_bar[stage], kb * BK, pe * 2 * p.f + p.f + feat);
-          } else if constexpr (MODE == kFwd2) {
-#pragma unroll
-            for (int i = 0; i < 2; ++i)
-              tc::tma_load_2d_pair(sB + i * kMnBlockBytes, &tmB, &full_bar[stage], kb * BK,
-                                   pe * p.Ndim + t.nt * BN + rank * (BN / 2) + 64 * i);
-          } else {
-#pragma unroll
-            for (int i = 0; i < 2; ++i)
-              tc::tma_load_2d_pair(sB + i * kMnBlockBytes, &tmB, &full_bar[stage],
-                                   t.nt * BN + rank * (BN / 2) + 64 * i, pe * p.Kdim + kb * BK);
+          if constexpr (MODE == kFwd1) {           // 64 gate features and the same 64 up features: W_gu as [2M][f][d]
+            tc::tma_load_3d_pair(sB, &tmB, &full_bar[stage], kb * BK, t.nt * (BN / 2) + rank * 64, 2 * pe);
+          } else if constexpr (MODE == kFwd2) {    // 128 rows of W_down
+            tc::tma_load_2d_pair(sB, &tmB, &full_bar[stage], kb * BK, pe * p.Ndim + t.nt * BN + rank * (BN / 2));
+          } else {                                 // two 64-column blocks of W_gu
+            tc::tma_load_3d_pair(sB, &tmB, &full_bar[stage], 0, pe * p.Kdim + kb * BK, t.nt * 4 + rank * 2);
           }
           if (++stage == kRowPairStages) { stage = 0; phase ^= 1u; }
         }
@@ -1165,12 +1164,12 @@ row_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 }
 
 template <int MODE>
-int launch(unipool_ctx* ctx, int phase, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC0,
-           const CUtensorMap& tmC1, const GemmParams& p, cudaStream_t s) {
+int launch(unipool_ctx* ctx, int phase, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB64,
+           const CUtensorMap& tmC0, const CUtensorMap& tmC1, const GemmParams& p, cudaStream_t s) {
   PhaseTimer pt(ctx, phase, 1, s);
   auto kern = grouped_gemm_tc_kernel<MODE>;
   UP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemTotal));
-  kern<<<ctx->sm_count, Traits<MODE>::kThreads, kSmemTotal, s>>>(tmA, tmB, tmC0, tmC1, p);
+  kern<<<ctx->sm_count, Traits<MODE>::kThreads, kSmemTotal, s>>>(tmA, tmB, tmB64, tmC0, tmC1, p);
   UP_LAUNCH_CHECK();
   return UNIPOOL_OK;
 }
@@ -1187,12 +1186,13 @@ bool rows_on_pairs(const unipool_ctx* ctx, int n_experts) {
   return (int64_t)ctx->cfg.max_tokens * ctx->cfg.top_k >= (int64_t)4 * BM * n_experts;
 }
 
-// One row-tile GEMM.  tmA / tmB: the operand maps of the single-CTA kernel; tmA64 / tmBp: those of the
-// pair kernel's half pair-tiles (64-row boxes of A) and of its B halves (64-row boxes).
+// One row-tile GEMM.  tmA / tmB / tmB64: the operand maps of the single-CTA kernel (tmB64: 64 x 64 boxes
+// of the weights for the column slices of the second dgrad); tmA64 / tmBp: those of the pair kernel's
+// half pair-tiles (64-row boxes of A) and of its B halves.
 template <int MODE>
 int launch_rows(unipool_ctx* ctx, int phase, bool pairs, const CUtensorMap& tmA, const CUtensorMap& tmA64,
-                const CUtensorMap& tmB, const CUtensorMap& tmBp, const CUtensorMap& tmC0, const CUtensorMap& tmC1,
-                const GemmParams& p, cudaStream_t s) {
+                const CUtensorMap& tmB, const CUtensorMap& tmB64, const CUtensorMap& tmBp, const CUtensorMap& tmC0,
+                const CUtensorMap& tmC1, const GemmParams& p, cudaStream_t s) {
   PhaseTimer pt(ctx, phase, 1, s);
   if (pairs) {
     auto kern = row_pair_kernel<MODE>;
@@ -1201,16 +1201,16 @@ int launch_rows(unipool_ctx* ctx, int phase, bool pairs, const CUtensorMap& tmA,
   } else {
     auto kern = grouped_gemm_tc_kernel<MODE>;
     UP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemTotal));
-    kern<<<ctx->sm_count, Traits<MODE>::kThreads, kSmemTotal, s>>>(tmA, tmB, tmC0, tmC1, p);
+    kern<<<ctx->sm_count, Traits<MODE>::kThreads, kSmemTotal, s>>>(tmA, tmB, tmB64, tmC0, tmC1, p);
   }
   UP_LAUNCH_CHECK();
   return UNIPOOL_OK;
 }
 
-// The pool weight gradient runs on CTA pairs (a device with a single SM falls back to the single-CTA kernel).
+// The pool weight gradient runs on CTA pairs.
 int launch_wgrad(unipool_ctx* ctx, int phase, const CUtensorMap& tmP, const CUtensorMap& tmQ, const CUtensorMap& tmW,
                  const GemmParams& p, cudaStream_t s) {
-  if (ctx->sm_count < 2) return launch<kWgrad>(ctx, phase, tmP, tmQ, tmW, tmW, p, s);
+  UP_REQUIRE(ctx->sm_count >= 2, UNIPOOL_ERR_UNSUPPORTED, "the weight gradient needs a device with CTA pairs");
   PhaseTimer pt(ctx, phase, 1, s);
   UP_CUDA(cudaFuncSetAttribute(wgrad_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPairSmemTotal));
   wgrad_pair_kernel<<<ctx->sm_count / 2 * 2, kThreads, kPairSmemTotal, s>>>(tmP, tmQ, tmW, p);
@@ -1232,16 +1232,16 @@ int wgrad_pair(unipool_ctx* ctx, const PoolWgradArgs& a, cudaStream_t s) {
   CUtensorMap tmP, tmQ, tmW;
   int rc;
   if (a.dW_down != nullptr) {                     // dW_down[e] [d, f] (+)= dYp_e^T A_e
-    if ((rc = map_2d(ctx, &tmP, a.dYp, d, rows, 64, 64)) != UNIPOOL_OK) return rc;
-    if ((rc = map_2d(ctx, &tmQ, a.A, f, rows, 64, 64)) != UNIPOOL_OK) return rc;
+    if ((rc = map_mn(ctx, &tmP, a.dYp, d, rows, 2)) != UNIPOOL_OK) return rc;
+    if ((rc = map_mn(ctx, &tmQ, a.A, f, rows, 2)) != UNIPOOL_OK) return rc;
     if ((rc = map_chunk(ctx, &tmW, a.dW_down, f, (uint64_t)M * d, kMapF32Chunk)) != UNIPOOL_OK) return rc;
     p.Mdim = d; p.Ndim = f;
     if ((rc = launch_wgrad(ctx, UNIPOOL_PH_WGRAD_DOWN, tmP, tmQ, tmW, p, s)) != UNIPOOL_OK) return rc;
   }
   if (a.dW_gu == nullptr) return UNIPOOL_OK;
   // dW_gu[e] [2f, d] (+)= dGU_e^T Xp_e
-  if ((rc = map_2d(ctx, &tmP, a.dGU, 2 * f, rows, 64, 64)) != UNIPOOL_OK) return rc;
-  if ((rc = map_2d(ctx, &tmQ, a.Xp, d, rows, 64, 64)) != UNIPOOL_OK) return rc;
+  if ((rc = map_mn(ctx, &tmP, a.dGU, 2 * f, rows, 2)) != UNIPOOL_OK) return rc;
+  if ((rc = map_mn(ctx, &tmQ, a.Xp, d, rows, 2)) != UNIPOOL_OK) return rc;
   if ((rc = map_chunk(ctx, &tmW, a.dW_gu, d, (uint64_t)M * 2 * f, kMapF32Chunk)) != UNIPOOL_OK) return rc;
   p.Mdim = 2 * f; p.Ndim = d;
   return launch_wgrad(ctx, UNIPOOL_PH_WGRAD_GU, tmP, tmQ, tmW, p, s);
@@ -1284,27 +1284,27 @@ int expert_fwd_tc(unipool_ctx* ctx, const ExpertFwdArgs& a, cudaStream_t s) {
   // 128 rows of W_gu viewed as [2M f, d]).
   if ((rc = map_2d(ctx, &tmA, a.Xp, d, cap, 64, BM)) != UNIPOOL_OK) return rc;
   if ((rc = map_2d(ctx, &tmA64, a.Xp, d, cap, 64, 64)) != UNIPOOL_OK) return rc;
-  if ((rc = map_2d(ctx, &tmBp, a.W_gu, d, (uint64_t)M * 2 * f, 64, 64)) != UNIPOOL_OK) return rc;
   {
     const uint64_t dims[3] = {(uint64_t)d, (uint64_t)f, (uint64_t)2 * M};
     const uint64_t strides[2] = {(uint64_t)d, (uint64_t)f * d};
-    const uint32_t box[3] = {64, BN / 2, 2};
+    const uint32_t box[3] = {64, BN / 2, 2}, box_pair[3] = {64, BN / 4, 2};
     if ((rc = make_tmap(ctx, &tmB, kMapOperand, a.W_gu, 3, dims, strides, box)) != UNIPOOL_OK) return rc;
+    if ((rc = make_tmap(ctx, &tmBp, kMapOperand, a.W_gu, 3, dims, strides, box_pair)) != UNIPOOL_OK) return rc;
   }
   if ((rc = map_chunk(ctx, &tmC0, a.GU, 2 * f, cap, kMapBf16Chunk)) != UNIPOOL_OK) return rc;
   if ((rc = map_chunk(ctx, &tmC1, a.A, f, cap, kMapBf16Chunk)) != UNIPOOL_OK) return rc;
   p.Ndim = f; p.Kdim = d;
-  if ((rc = launch_rows<kFwd1>(ctx, UNIPOOL_PH_EXPERT_FWD_GU, plan, tmA, tmA64, tmB, tmBp, tmC0, tmC1, p, s)) != UNIPOOL_OK)
+  if ((rc = launch_rows<kFwd1>(ctx, UNIPOOL_PH_EXPERT_FWD_GU, plan, tmA, tmA64, tmB, tmB, tmBp, tmC0, tmC1, p, s)) != UNIPOOL_OK)
     return rc;
   // Yp = A W_down^T
   if ((rc = map_2d(ctx, &tmA, a.A, f, cap, 64, BM)) != UNIPOOL_OK) return rc;
   if ((rc = map_2d(ctx, &tmA64, a.A, f, cap, 64, 64)) != UNIPOOL_OK) return rc;
   if ((rc = map_2d(ctx, &tmB, a.W_down, f, (uint64_t)M * d, 64, BN)) != UNIPOOL_OK) return rc;
-  if ((rc = map_2d(ctx, &tmBp, a.W_down, f, (uint64_t)M * d, 64, 64)) != UNIPOOL_OK) return rc;   // 64-row boxes
-  tmC1 = tmBp;                                                                                    // column slices
+  if ((rc = map_2d(ctx, &tmBp, a.W_down, f, (uint64_t)M * d, 64, BN / 2)) != UNIPOOL_OK) return rc;   // a CTA's half
+  if ((rc = map_2d(ctx, &tmC1, a.W_down, f, (uint64_t)M * d, 64, 64)) != UNIPOOL_OK) return rc;       // column slices
   if ((rc = map_chunk(ctx, &tmC0, a.Yp, d, cap, kMapBf16Chunk)) != UNIPOOL_OK) return rc;
   p.Ndim = d; p.Kdim = f;
-  return launch_rows<kFwd2>(ctx, UNIPOOL_PH_EXPERT_FWD_DOWN, plan, tmA, tmA64, tmB, tmBp, tmC0, tmC1, p, s);
+  return launch_rows<kFwd2>(ctx, UNIPOOL_PH_EXPERT_FWD_DOWN, plan, tmA, tmA64, tmB, tmB, tmBp, tmC0, tmC1, p, s);
 }
 
 int expert_bwd_tc(unipool_ctx* ctx, const ExpertBwdArgs& a, cudaStream_t s) {
@@ -1317,24 +1317,28 @@ int expert_bwd_tc(unipool_ctx* ctx, const ExpertBwdArgs& a, cudaStream_t s) {
   p.expert_base = a.expert_base;
   p.f = f;
   p.status = ctx->ws.status;
-  CUtensorMap tmA, tmB, tmC0, tmC1;
+  CUtensorMap tmA, tmB, tmB64, tmBp, tmC0, tmC1;
   int rc;
   // dA = dYp W_down, fused with the SwiGLU derivative -> dGU
   if ((rc = map_2d(ctx, &tmA, a.dYp, d, cap, 64, BM)) != UNIPOOL_OK) return rc;
-  if ((rc = map_2d(ctx, &tmB, a.W_down, f, (uint64_t)M * d, 64, 64)) != UNIPOOL_OK) return rc;
+  if ((rc = map_mn(ctx, &tmB, a.W_down, f, (uint64_t)M * d, BN / 64)) != UNIPOOL_OK) return rc;
+  if ((rc = map_2d(ctx, &tmB64, a.W_down, f, (uint64_t)M * d, 64, 64)) != UNIPOOL_OK) return rc;
   if ((rc = map_chunk(ctx, &tmC0, a.dGU, 2 * f, cap, kMapBf16Chunk)) != UNIPOOL_OK) return rc;
   if ((rc = map_chunk(ctx, &tmC1, a.GU, 2 * f, cap, kMapBf16Chunk)) != UNIPOOL_OK) return rc;
   p.Ndim = f; p.Kdim = d;
-  if ((rc = launch<kDgrad1>(ctx, UNIPOOL_PH_DGRAD_DOWN, tmA, tmB, tmC0, tmC1, p, s)) != UNIPOOL_OK) return rc;
+  if ((rc = launch<kDgrad1>(ctx, UNIPOOL_PH_DGRAD_DOWN, tmA, tmB, tmB64, tmC0, tmC1, p, s)) != UNIPOOL_OK) return rc;
   // dXp = dGU [W_gate; W_up]
   if ((rc = map_2d(ctx, &tmA, a.dGU, 2 * f, cap, 64, BM)) != UNIPOOL_OK) return rc;
-  if ((rc = map_2d(ctx, &tmB, a.W_gu, d, (uint64_t)M * 2 * f, 64, 64)) != UNIPOOL_OK) return rc;
+  if ((rc = map_mn(ctx, &tmB, a.W_gu, d, (uint64_t)M * 2 * f, BN / 64)) != UNIPOOL_OK) return rc;
+  if ((rc = map_mn(ctx, &tmBp, a.W_gu, d, (uint64_t)M * 2 * f, BN / 128)) != UNIPOOL_OK) return rc;
+  if ((rc = map_2d(ctx, &tmB64, a.W_gu, d, (uint64_t)M * 2 * f, 64, 64)) != UNIPOOL_OK) return rc;
   if ((rc = map_chunk(ctx, &tmC0, a.dXp, d, cap, kMapBf16Chunk)) != UNIPOOL_OK) return rc;
   p.Ndim = d; p.Kdim = 2 * f; p.overwrite = 1;
   p.group_offsets = a.offsets;
   CUtensorMap tmA64;
   if ((rc = map_2d(ctx, &tmA64, a.dGU, 2 * f, cap, 64, 64)) != UNIPOOL_OK) return rc;
-  rc = launch_rows<kDgrad2>(ctx, UNIPOOL_PH_DGRAD_GU, rows_on_pairs(ctx, a.n_experts), tmA, tmA64, tmB, tmB, tmC0, tmC0, p, s);
+  rc = launch_rows<kDgrad2>(ctx, UNIPOOL_PH_DGRAD_GU, rows_on_pairs(ctx, a.n_experts), tmA, tmA64, tmB, tmB64, tmBp, tmC0,
+                            tmC0, p, s);
   if (rc != UNIPOOL_OK) return rc;
   if (a.wgrad) {
     PoolWgradArgs w{1, 0, a.offsets, a.Xp, a.A, a.dYp, a.dGU, a.expert_base, a.n_experts, a.dW_gu, a.dW_down,
@@ -1365,13 +1369,14 @@ int router_bwd_gemms_tc(unipool_ctx* ctx, const void* dz16, int Mp, const void* 
   GemmParams p{};
   p.status = ctx->ws.status;
   p.n_experts = 1;
-  CUtensorMap tmA, tmB, tmC;
+  CUtensorMap tmA, tmB, tmB64, tmC;
   int rc;
   if ((rc = map_2d(ctx, &tmA, dz16, Mp, T, 64, BM)) != UNIPOOL_OK) return rc;
-  if ((rc = map_2d(ctx, &tmB, W16, d, M, 64, 64)) != UNIPOOL_OK) return rc;
+  if ((rc = map_mn(ctx, &tmB, W16, d, M, BN / 64)) != UNIPOOL_OK) return rc;
+  if ((rc = map_2d(ctx, &tmB64, W16, d, M, 64, 64)) != UNIPOOL_OK) return rc;
   if ((rc = map_chunk(ctx, &tmC, dx, d, T, kMapBf16Chunk)) != UNIPOOL_OK) return rc;
   p.Mdim = (T + BM - 1) / BM; p.Ndim = d; p.Kdim = Mp; p.overwrite = 0;
-  if ((rc = launch<kDgrad2>(ctx, UNIPOOL_PH_ROUTE_BWD_DX, tmA, tmB, tmC, tmC, p, s)) != UNIPOOL_OK) return rc;
+  if ((rc = launch<kDgrad2>(ctx, UNIPOOL_PH_ROUTE_BWD_DX, tmA, tmB, tmB64, tmC, tmC, p, s)) != UNIPOOL_OK) return rc;
 
   const int out_tiles = ((M + BM - 1) / BM) * ((d + BN - 1) / BN);
   const int t64 = (T + 63) / 64;
@@ -1380,12 +1385,12 @@ int router_bwd_gemms_tc(unipool_ctx* ctx, const void* dz16, int Mp, const void* 
   if (splits > t64) splits = t64;
   const int chunk = ((t64 + splits - 1) / splits) * 64;
   splits = (t64 * 64 + chunk - 1) / chunk;
-  if ((rc = map_2d(ctx, &tmA, dz16, Mp, T, 64, 64)) != UNIPOOL_OK) return rc;
-  if ((rc = map_2d(ctx, &tmB, x, d, T, 64, 64)) != UNIPOOL_OK) return rc;
+  if ((rc = map_mn(ctx, &tmA, dz16, Mp, T, BM / 64)) != UNIPOOL_OK) return rc;
+  if ((rc = map_mn(ctx, &tmB, x, d, T, BN / 64)) != UNIPOOL_OK) return rc;
   if ((rc = map_chunk(ctx, &tmC, dW_r, d, M, kMapF32Chunk)) != UNIPOOL_OK) return rc;
   p.n_experts = splits; p.n_layers = 1; p.uniform_rows = t64 * 64;
   p.Mdim = M; p.Ndim = d; p.Kdim = chunk; p.overwrite = 0;
-  return launch<kWgrad>(ctx, UNIPOOL_PH_ROUTE_BWD_DW, tmA, tmB, tmC, tmC, p, s);
+  return launch<kWgrad>(ctx, UNIPOOL_PH_ROUTE_BWD_DW, tmA, tmB, tmB, tmC, tmC, p, s);
 }
 
 }  // namespace unipool
