@@ -43,7 +43,7 @@ NCU_TRAFFIC = {("182m", "expert_fwd_gu"): 4 * (165.59e6 + 78.63e6)}
 GEMM_KERNEL = {"expert_fwd_gu": "grouped_gemm_tc_kernel", "expert_fwd_down": "grouped_gemm_tc_kernel",
                "dgrad_down": "grouped_gemm_tc_kernel", "dgrad_gu": "grouped_gemm_tc_kernel",
                "wgrad_down": "wgrad_pair_kernel", "wgrad_gu": "wgrad_pair_kernel"}
-DISPATCH_MAP_LAUNCHES = 3
+DISPATCH_MAP_LAUNCHES = 1
 
 METRIC = "moe_layer_fwd_bwd_tokens_per_s"
 UNIT = "tokens/s"

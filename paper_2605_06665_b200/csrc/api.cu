@@ -39,7 +39,7 @@ Workspace carve_workspace(const unipool_config& cfg, void* base) {
   };
   const size_t eb = cfg.dtype == UNIPOOL_BF16 ? 2 : 4;
   const int64_t cap = row_capacity_of(cfg);
-  const int64_t blocks = ((int64_t)cfg.max_tokens + kDispatchChunkTokens - 1) / kDispatchChunkTokens;
+  const int64_t blocks = ((int64_t)cfg.max_tokens + kDispatchMinChunkTokens - 1) / kDispatchMinChunkTokens;
   w.status = reinterpret_cast<int32_t*>(take(4 * sizeof(int32_t)));
   w.route_counts = reinterpret_cast<int32_t*>(take(UNIPOOL_MAX_EXPERTS * sizeof(int32_t)));
   w.route_sums = reinterpret_cast<double*>(take(UNIPOOL_MAX_EXPERTS * sizeof(double)));

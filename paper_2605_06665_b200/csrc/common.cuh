@@ -62,7 +62,8 @@ struct Workspace {
   size_t   bytes;         // total
 };
 
-constexpr int kDispatchChunkTokens = 256;  // tokens per dispatch block (eight warps of 32 tokens)
+constexpr int kDispatchChunkTokens = 256;     // most tokens per block of the permute kernels (eight warps of 32)
+constexpr int kDispatchMinChunkTokens = 64;   // fewest
 
 Workspace carve_workspace(const unipool_config& cfg, void* base);
 

@@ -10,18 +10,19 @@ namespace unipool {
 // Block b owns tokens [b*CH, (b+1)*CH), warp w of it the tokens [w*CH/8, (w+1)*CH/8) of those: the
 // stable (token-major) order is block order, then warp order, then lane order inside a warp.
 constexpr int kDispatchWarps = 8;
-constexpr int kDispatchWarpTokens = kDispatchChunkTokens / kDispatchWarps;
+// A chunk holds `chunk` tokens (a multiple of 8, at most kDispatchChunkTokens), a warp chunk / 8 of them.
 
 // hist[w][e] = assignments to expert e among warp w's tokens (shared memory, [kDispatchWarps][M]).
 // `status` (may be NULL) receives a corrupt routing entry; the assignment is dropped either way.
-__device__ __forceinline__ void chunk_histograms(const int32_t* __restrict__ idx, int T, int k, int M, int* hist,
-                                                 int32_t* status, int64_t& a_begin, int64_t& a_end) {
+__device__ __forceinline__ void chunk_histograms(const int32_t* __restrict__ idx, int T, int k, int M, int chunk,
+                                                 int* hist, int32_t* status, int64_t& a_begin, int64_t& a_end) {
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
   for (int i = threadIdx.x; i < kDispatchWarps * M; i += blockDim.x) hist[i] = 0;
   __syncthreads();
   const int64_t total = (int64_t)T * k;
-  a_begin = min(total, ((int64_t)blockIdx.x * kDispatchChunkTokens + (int64_t)warp * kDispatchWarpTokens) * k);
-  a_end = min(total, a_begin + (int64_t)kDispatchWarpTokens * k);
+  const int warp_tokens = chunk / kDispatchWarps;
+  a_begin = min(total, ((int64_t)blockIdx.x * chunk + (int64_t)warp * warp_tokens) * k);
+  a_end = min(total, a_begin + (int64_t)warp_tokens * k);
   for (int64_t a = a_begin + lane; a < a_end; a += 32) {
     const int e = idx[a];
     if (e < 0 || e >= M) {          // corrupt routing table: record it, drop the assignment
@@ -34,94 +35,92 @@ __device__ __forceinline__ void chunk_histograms(const int32_t* __restrict__ idx
 }
 
 __global__ void __launch_bounds__(kDispatchWarps * 32)
-dispatch_hist_kernel(const int32_t* __restrict__ idx, int T, int k, int M, int32_t* __restrict__ block_hist,
-                     int32_t* __restrict__ status) {
+dispatch_hist_kernel(const int32_t* __restrict__ idx, int T, int k, int M, int chunk,
+                     int32_t* __restrict__ block_hist, int32_t* __restrict__ status) {
   extern __shared__ int hist[];
   int64_t a_begin, a_end;
-  chunk_histograms(idx, T, k, M, hist, status, a_begin, a_end);
+  chunk_histograms(idx, T, k, M, chunk, hist, status, a_begin, a_end);
   for (int e = threadIdx.x; e < M; e += blockDim.x) {
     int total = 0;
 #pragma unroll
     for (int w = 0; w < kDispatchWarps; ++w) total += hist[w * M + e];
-    block_hist[(int64_t)blockIdx.x * M + e] = total;
+    block_hist[(int64_t)e * gridDim.x + blockIdx.x] = total;      // expert-major: [M][chunks]
   }
 }
 
-// One block of 1024 threads: per-expert totals -> padded exclusive scan -> per-(chunk, expert) bases.
-// block_hist[b][e] is replaced by the first row of chunk b's assignments to e.  Thread (seg, e)
-// walks a contiguous segment of chunks for expert e, so that the loads of one pass are independent
-// and coalesced over e.
-constexpr int kScanThreads = 1024;
-__global__ void __launch_bounds__(kScanThreads)
-dispatch_scan_kernel(int32_t* __restrict__ block_hist, int n_blocks, int M, int row_capacity,
-                     int32_t* __restrict__ offsets, int32_t* __restrict__ token_of,
-                     int32_t* __restrict__ tile_expert) {
-  __shared__ int part[kScanThreads];                  // [segs][M] chunk-segment sums, then bases
-  __shared__ int start[UNIPOOL_MAX_EXPERTS + 1];
-  __shared__ int total_s[UNIPOOL_MAX_EXPERTS];
-  const int segs = kScanThreads / M < 1 ? 1 : (kScanThreads / M > 32 ? 32 : kScanThreads / M);
-  const int per_seg = (n_blocks + segs - 1) / segs;
-  const int e = threadIdx.x % M, seg = threadIdx.x / M;
-  const bool worker = seg < segs;
-  const int b0 = seg * per_seg, b1 = min(n_blocks, b0 + per_seg);
-  if (worker) {
-    int sum = 0;
-#pragma unroll 8
-    for (int b = b0; b < b1; ++b) sum += block_hist[(int64_t)b * M + e];
-    part[seg * M + e] = sum;
-  }
-  __syncthreads();
-  if (threadIdx.x < M) {                               // totals and segment bases of expert threadIdx.x
-    int run = 0;
-    for (int sg = 0; sg < segs; ++sg) { const int v = part[sg * M + threadIdx.x]; part[sg * M + threadIdx.x] = run; run += v; }
-    total_s[threadIdx.x] = run;
-  }
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    int run = 0;
-    for (int i = 0; i < M; ++i) {
-      start[i] = run;
-      run += (total_s[i] + UNIPOOL_ROW_ALIGN - 1) / UNIPOOL_ROW_ALIGN * UNIPOOL_ROW_ALIGN;
-    }
-    start[M] = run;
-  }
-  __syncthreads();
-  if (threadIdx.x <= M) offsets[threadIdx.x] = start[threadIdx.x];
-  if (worker) {
-    int run = start[e] + part[seg * M + e];
-#pragma unroll 8
-    for (int b = b0; b < b1; ++b) {
-      const int h = block_hist[(int64_t)b * M + e];
-      block_hist[(int64_t)b * M + e] = run;
-      run += h;
-    }
-  }
-  // pad rows of every group, rows beyond the last group, tile -> expert table
-  const int used = start[M];
-  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-  for (int g = warp; g < M; g += kScanThreads / 32) {
-    const int lo = start[g] + total_s[g], hi = start[g + 1];
-    for (int r = lo + lane; r < hi; r += 32) token_of[r] = -1;
-    for (int tl = start[g] / UNIPOOL_ROW_ALIGN + lane; tl < hi / UNIPOOL_ROW_ALIGN; tl += 32) tile_expert[tl] = g;
-  }
-  for (int r = used + threadIdx.x; r < row_capacity; r += blockDim.x) token_of[r] = -1;
-  for (int tl = used / UNIPOOL_ROW_ALIGN + threadIdx.x; tl < row_capacity / UNIPOOL_ROW_ALIGN; tl += blockDim.x)
-    tile_expert[tl] = -1;
-}
+// Second (and last) kernel of the permute.  Block b owns the tokens of chunk b.  From the per-chunk
+// histograms of the first kernel every block derives, for itself, the padded group starts (column sums
+// over all chunks, exclusive scan over the experts) and the rows its own chunk starts at (column sums
+// over the chunks before it); it then ranks its assignments (block, warp, lane order = token order, so
+// the permutation is stable), writes row_of / token_of and moves its tokens: a token's row is read
+// once and written to each of its k rows.  Every block also takes a share of the bookkeeping: pad rows
+// (token_of = -1, zeros in Xp), the tile -> expert table, the rows behind the last group.
+constexpr int kPlaceTokens = 8;          // tokens a warp has in flight while moving rows
+constexpr int kVpl = 3;                  // 16-byte vectors per lane and pass of the row movers
 
-// block_base[b][e] = first row of block b's assignments to expert e (written by the scan).  The
-// block rebuilds its warps' histograms, turns them into each warp's first row per expert, and every
-// warp ranks its assignments in lane order.
 __global__ void __launch_bounds__(kDispatchWarps * 32)
-dispatch_rank_kernel(const int32_t* __restrict__ idx, int T, int k, int M,
-                     const int32_t* __restrict__ block_base, int32_t* __restrict__ row_of,
-                     int32_t* __restrict__ token_of) {
-  extern __shared__ int hist[];
+dispatch_place_kernel(const int32_t* __restrict__ idx, int T, int k, int M, int chunk,
+                      const int32_t* __restrict__ block_hist, int n_blocks, const uint4* __restrict__ x,
+                      int row_vecs, int row_capacity, int32_t* __restrict__ offsets,
+                      int32_t* __restrict__ row_of, int32_t* __restrict__ token_of,
+                      int32_t* __restrict__ tile_expert, uint4* __restrict__ Xp) {
+  extern __shared__ int sm[];
+  int* hist = sm;                                   // [8][M] per-warp histograms, then per-warp next rows
+  int* start = hist + kDispatchWarps * M;           // [M + 1] group starts
+  int* total = start + M + 1;                       // [M] assignments per expert, all chunks
+  int* before = total + M;                          // [M] assignments per expert in the chunks before this one
+  int* rows_s = before + M;                         // [chunk * k] row of each assignment of this chunk
+  __shared__ int warp_sum[kDispatchWarps];
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+  const int me = (int)blockIdx.x;
+
+  // (a) sums over the chunks of the (expert-major) chunk histograms: a warp per expert, lanes over chunks
+  for (int e = warp; e < M; e += kDispatchWarps) {
+    int tot = 0, bef = 0;
+    for (int b = lane; b < n_blocks; b += 32) {
+      const int v = block_hist[(int64_t)e * n_blocks + b];
+      tot += v;
+      bef += b < me ? v : 0;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      tot += __shfl_xor_sync(0xffffffffu, tot, o);
+      bef += __shfl_xor_sync(0xffffffffu, bef, o);
+    }
+    if (lane == 0) { total[e] = tot; before[e] = bef; }
+  }
+  __syncthreads();
+  // (b) exclusive scan of the padded totals: a thread takes a run of experts, warps and the block scan the runs
+  {
+    const int per = (M + (int)blockDim.x - 1) / (int)blockDim.x;
+    const int e0 = threadIdx.x * per;
+    int mine = 0;
+    for (int i = 0; i < per; ++i)
+      if (e0 + i < M) mine += (total[e0 + i] + UNIPOOL_ROW_ALIGN - 1) / UNIPOOL_ROW_ALIGN * UNIPOOL_ROW_ALIGN;
+    int incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += v;
+    }
+    if (lane == 31) warp_sum[warp] = incl;
+    __syncthreads();
+    int base = 0;
+    for (int w = 0; w < warp; ++w) base += warp_sum[w];
+    int run = base + incl - mine;
+    for (int i = 0; i < per; ++i)
+      if (e0 + i < M) {
+        start[e0 + i] = run;
+        run += (total[e0 + i] + UNIPOOL_ROW_ALIGN - 1) / UNIPOOL_ROW_ALIGN * UNIPOOL_ROW_ALIGN;
+      }
+    if (threadIdx.x == blockDim.x - 1) start[M] = run;   // the last thread's run ends the last group
+  }
+  __syncthreads();
+  // (c) this chunk's per-warp histograms -> first row of every warp per expert
   int64_t a_begin, a_end;
-  chunk_histograms(idx, T, k, M, hist, nullptr, a_begin, a_end);
+  chunk_histograms(idx, T, k, M, chunk, hist, nullptr, a_begin, a_end);
   for (int e = threadIdx.x; e < M; e += blockDim.x) {
-    int run = block_base[(int64_t)blockIdx.x * M + e];
+    int run = start[e] + before[e];
 #pragma unroll
     for (int w = 0; w < kDispatchWarps; ++w) {
       const int n = hist[w * M + e];
@@ -130,6 +129,8 @@ dispatch_rank_kernel(const int32_t* __restrict__ idx, int T, int k, int M,
     }
   }
   __syncthreads();
+  // (d) ranks: every warp walks its assignments in lane order
+  const int64_t chunk_a0 = (int64_t)me * chunk * k;
   int* next_row = hist + warp * M;
   for (int64_t a0 = a_begin; a0 < a_end; a0 += 32) {
     const int64_t a = a0 + lane;
@@ -144,41 +145,57 @@ dispatch_rank_kernel(const int32_t* __restrict__ idx, int T, int k, int M,
     __syncwarp();
     if (ok && rank == 0) next_row[e] += __popc(peers);       // leader = lowest lane of the peer set
     __syncwarp();
-    if (live) row_of[a] = row;
+    if (live) { row_of[a] = row; rows_s[a - chunk_a0] = row; }
     if (ok) token_of[row] = (int)(a / k);
   }
-}
-
-// ---------------------------------------------------------------- row movers
-// One warp moves one row in 16-byte vectors; a lane owns vectors lane, lane + 32, ... and issues
-// all loads of a pass (kVpl vectors per lane and source row) before it uses any of them.
-constexpr int kVpl = 3;
-
-// Xp[r] = x[token_of[r]]  (zero on pad rows), rows < offsets[M].
-__global__ void __launch_bounds__(256)
-gather_rows_kernel(const uint4* __restrict__ x, const int32_t* __restrict__ token_of,
-                   const int32_t* __restrict__ offsets_end, uint4* __restrict__ Xp, int row_vecs,
-                   int row_capacity) {
-  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-  const int used = *offsets_end;
-  for (int r = blockIdx.x * 8 + warp; r < used; r += gridDim.x * 8) {
-    const int t = token_of[r];
-    uint4* dst = Xp + (int64_t)r * row_vecs;
-    const uint4* src = x + (int64_t)(t >= 0 ? t : 0) * row_vecs;
-    for (int v0 = lane; v0 < row_vecs; v0 += 32 * kVpl) {
-      uint4 buf[kVpl];
+  __syncthreads();
+  // (e) move the chunk's tokens: a warp keeps kPlaceTokens rows of x in flight
+  const int t0 = me * chunk;
+  const int n_tok = min(chunk, T - t0);
+  for (int v0 = lane; v0 < row_vecs; v0 += 32 * kVpl) {
+    for (int tt = warp * kPlaceTokens; tt < n_tok; tt += kDispatchWarps * kPlaceTokens) {
+      uint4 buf[kPlaceTokens][kVpl];
 #pragma unroll
-      for (int i = 0; i < kVpl; ++i) {
-        const int v = v0 + 32 * i;
-        buf[i] = (t >= 0 && v < row_vecs) ? __ldg(src + v) : make_uint4(0, 0, 0, 0);
-      }
+      for (int q = 0; q < kPlaceTokens; ++q)
 #pragma unroll
-      for (int i = 0; i < kVpl; ++i) {
-        const int v = v0 + 32 * i;
-        if (v < row_vecs) dst[v] = buf[i];
+        for (int i = 0; i < kVpl; ++i) {
+          const int v = v0 + 32 * i;
+          buf[q][i] = (tt + q < n_tok && v < row_vecs) ? __ldg(x + (int64_t)(t0 + tt + q) * row_vecs + v)
+                                                       : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+      for (int q = 0; q < kPlaceTokens; ++q) {
+        if (tt + q >= n_tok) break;
+        for (int j = 0; j < k; ++j) {
+          const int row = rows_s[(tt + q) * k + j];
+          if (row < 0) continue;
+          uint4* dst = Xp + (int64_t)row * row_vecs;
+#pragma unroll
+          for (int i = 0; i < kVpl; ++i) {
+            const int v = v0 + 32 * i;
+            if (v < row_vecs) dst[v] = buf[q][i];
+          }
+        }
       }
     }
   }
+  // (f) bookkeeping, shared out over the blocks
+  if (me == 0)
+    for (int e = threadIdx.x; e <= M; e += blockDim.x) offsets[e] = start[e];
+  for (int e = me; e < M; e += gridDim.x) {
+    const int lo = start[e] + total[e], hi = start[e + 1];
+    for (int r = lo + warp; r < hi; r += kDispatchWarps) {               // pad rows: no token, zeros
+      if (lane == 0) token_of[r] = -1;
+      uint4* dst = Xp + (int64_t)r * row_vecs;
+      for (int v = lane; v < row_vecs; v += 32) dst[v] = make_uint4(0, 0, 0, 0);
+    }
+    for (int tl = start[e] / UNIPOOL_ROW_ALIGN + threadIdx.x; tl < hi / UNIPOOL_ROW_ALIGN; tl += blockDim.x)
+      tile_expert[tl] = e;
+  }
+  const int used = start[M];
+  const int gid = me * (int)blockDim.x + threadIdx.x, gstride = (int)(gridDim.x * blockDim.x);
+  for (int r = used + gid; r < row_capacity; r += gstride) token_of[r] = -1;
+  for (int tl = used / UNIPOOL_ROW_ALIGN + gid; tl < row_capacity / UNIPOOL_ROW_ALIGN; tl += gstride) tile_expert[tl] = -1;
 }
 
 template <typename T> struct Vec16;
@@ -345,6 +362,19 @@ __global__ void dispatch_empty_kernel(int32_t* offsets, int32_t* token_of, int32
   if (i < row_capacity / UNIPOOL_ROW_ALIGN) tile_expert[i] = -1;
 }
 
+static size_t place_smem_bytes(int M, int k, int chunk) {
+  return ((size_t)kDispatchWarps * M + (M + 1) + 2 * (size_t)M + (size_t)chunk * k) * sizeof(int);
+}
+
+// Tokens per chunk (= per block of the two permute kernels): the largest of 256, 128, 64 that still
+// gives every SM a block - a block moves its own tokens, and an SM alone pulls well under its share of
+// the memory bandwidth; but every block reads the histograms of all chunks, so no more chunks than that.
+static int dispatch_chunk_tokens(int T, int sm_count) {
+  for (int chunk = kDispatchChunkTokens; chunk > kDispatchMinChunkTokens; chunk /= 2)
+    if ((T + chunk - 1) / chunk >= sm_count) return chunk;
+  return kDispatchMinChunkTokens;
+}
+
 static int row_mover_grid(const unipool_ctx* ctx, int64_t rows) {
   int64_t want = (rows + 7) / 8;
   int64_t cap = (int64_t)ctx->sm_count * 8;      // 8 resident 256-thread blocks per SM
@@ -361,21 +391,20 @@ int dispatch_launch(unipool_ctx* ctx, const void* x, int T, const int32_t* idx, 
     UP_LAUNCH_CHECK();
     return UNIPOOL_OK;
   }
-  const int n_blocks = (T + kDispatchChunkTokens - 1) / kDispatchChunkTokens;
+  const int chunk = dispatch_chunk_tokens(T, ctx->sm_count);
+  const int n_blocks = (T + chunk - 1) / chunk;
   int32_t* bh = ctx->ws.block_hist;
+  const int row_vecs = (int)((size_t)d * ctx->elem_bytes / 16);
   {
-  PhaseTimer pt(ctx, UNIPOOL_PH_DISPATCH_MAPS, 3, s);
-  dispatch_hist_kernel<<<n_blocks, kDispatchWarps * 32, kDispatchWarps * M * sizeof(int), s>>>(idx, T, k, M, bh, ctx->ws.status);
-  UP_LAUNCH_CHECK();
-  dispatch_scan_kernel<<<1, kScanThreads, 0, s>>>(bh, n_blocks, M, cap, offsets, token_of, tile_expert);
-  UP_LAUNCH_CHECK();
-  dispatch_rank_kernel<<<n_blocks, kDispatchWarps * 32, kDispatchWarps * M * sizeof(int), s>>>(idx, T, k, M, bh, row_of, token_of);
-  UP_LAUNCH_CHECK();
+    PhaseTimer pt(ctx, UNIPOOL_PH_DISPATCH_MAPS, 1, s);
+    dispatch_hist_kernel<<<n_blocks, kDispatchWarps * 32, kDispatchWarps * M * sizeof(int), s>>>(idx, T, k, M, chunk, bh,
+                                                                                                ctx->ws.status);
+    UP_LAUNCH_CHECK();
   }
   PhaseTimer pt(ctx, UNIPOOL_PH_DISPATCH_GATHER, 1, s);
-  const int row_vecs = (int)((size_t)d * ctx->elem_bytes / 16);
-  gather_rows_kernel<<<row_mover_grid(ctx, cap), 256, 0, s>>>(
-      static_cast<const uint4*>(x), token_of, offsets + M, static_cast<uint4*>(Xp), row_vecs, cap);
+  dispatch_place_kernel<<<n_blocks, kDispatchWarps * 32, place_smem_bytes(M, k, chunk), s>>>(
+      idx, T, k, M, chunk, bh, n_blocks, static_cast<const uint4*>(x), row_vecs, cap, offsets, row_of, token_of, tile_expert,
+      static_cast<uint4*>(Xp));
   UP_LAUNCH_CHECK();
   return UNIPOOL_OK;
 }
@@ -455,9 +484,9 @@ namespace {
 constexpr int64_t kStaticHistInts = 1024 * 512 - 64;      // chunks x experts that fit
 static __device__ __align__(256) int32_t g_dispatch_scratch[1024 * 512];
 constexpr int kMaxDevices = 64;
-// per device: the array's address there and the SM count, looked up by the first call on that device.
+// per device: the array's address there, looked up by the first call on that device.
 // Host threads may race on the first call: the entry is complete before its address becomes visible.
-struct ScratchInfo { int32_t* addr; int sms; };
+struct ScratchInfo { int32_t* addr; };
 std::atomic<const ScratchInfo*> g_scratch[kMaxDevices];
 ScratchInfo g_scratch_slots[kMaxDevices][2];
 std::atomic<int> g_scratch_next[kMaxDevices];
@@ -499,11 +528,9 @@ extern "C" int unipool_dispatch_static(const void* x, int32_t T, int32_t d_model
     // same values; each fills a slot of its own and publishes it.
     int32_t* ptr = nullptr;
     UP_CUDA(cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_dispatch_scratch));
-    int sms = 0;
-    UP_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    UP_REQUIRE(ptr != nullptr && sms > 0, UNIPOOL_ERR_CUDA, "dispatch_static: no address for the built-in scratch");
+    UP_REQUIRE(ptr != nullptr, UNIPOOL_ERR_CUDA, "dispatch_static: no address for the built-in scratch");
     const int slot = g_scratch_next[dev].fetch_add(1) & 1;
-    g_scratch_slots[dev][slot] = ScratchInfo{ptr, sms};
+    g_scratch_slots[dev][slot] = ScratchInfo{ptr};
     g_scratch[dev].store(&g_scratch_slots[dev][slot], std::memory_order_release);
     info = &g_scratch_slots[dev][slot];
   }
@@ -517,17 +544,13 @@ extern "C" int unipool_dispatch_static(const void* x, int32_t T, int32_t d_model
   }
   // the histograms are fully rewritten by the first kernel for the chunks of this call; nothing
   // else in the array has to start at zero
-  dispatch_hist_kernel<<<n_blocks, kDispatchWarps * 32, kDispatchWarps * n_experts * sizeof(int), s>>>(idx, T, top_k, n_experts, bh, status);
-  UP_LAUNCH_CHECK();
-  dispatch_scan_kernel<<<1, kScanThreads, 0, s>>>(bh, n_blocks, n_experts, cap, offsets, token_of, tile_expert);
-  UP_LAUNCH_CHECK();
-  dispatch_rank_kernel<<<n_blocks, kDispatchWarps * 32, kDispatchWarps * n_experts * sizeof(int), s>>>(idx, T, top_k, n_experts, bh, row_of, token_of);
+  dispatch_hist_kernel<<<n_blocks, kDispatchWarps * 32, kDispatchWarps * n_experts * sizeof(int), s>>>(
+      idx, T, top_k, n_experts, kDispatchChunkTokens, bh, status);
   UP_LAUNCH_CHECK();
   const int row_vecs = (int)((size_t)d_model * eb / 16);
-  int64_t want = ((int64_t)cap + 7) / 8, lim = (int64_t)info->sms * 8;
-  const int grid = (int)(want < 1 ? 1 : (want < lim ? want : lim));
-  gather_rows_kernel<<<grid, 256, 0, s>>>(static_cast<const uint4*>(x), token_of, offsets + n_experts,
-                                          static_cast<uint4*>(Xp), row_vecs, cap);
+  dispatch_place_kernel<<<n_blocks, kDispatchWarps * 32, place_smem_bytes(n_experts, top_k, kDispatchChunkTokens), s>>>(
+      idx, T, top_k, n_experts, kDispatchChunkTokens, bh, n_blocks, static_cast<const uint4*>(x), row_vecs, cap, offsets, row_of, token_of,
+      tile_expert, static_cast<uint4*>(Xp));
   UP_LAUNCH_CHECK();
   return UNIPOOL_OK;
 }
