@@ -35,9 +35,10 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of a workload's dominant kernel,
-# from the ncu capture summarised in profiles/grouped_gemm_182m_slice_ncu.txt: the 182m_slice case (a quarter
-# of the experts and of the rows of one 182m layer) moved 165.6 + 78.6 MB; a full launch is four times that.
-NCU_TRAFFIC = {("182m", "expert_fwd_gu"): 4 * (165.59e6 + 78.63e6)}
+# from the ncu capture summarised in profiles/grouped_gemm_978m_slice_ncu.txt: the 978m_slice case (an
+# eighth of the experts and of the rows of one 978m layer) moved 733.9 + 207.8 MB; a full launch is eight
+# times that (weights and activations both grow with the units processed).
+NCU_TRAFFIC = {("978m", "expert_fwd_gu"): 8 * (733.89e6 + 207.79e6)}
 
 # kernel behind each grouped-GEMM phase (for the roofline's `kernel` field) and launches of one dispatch-map call
 GEMM_KERNEL = {"expert_fwd_gu": "grouped_gemm_tc_kernel", "expert_fwd_down": "grouped_gemm_tc_kernel",
