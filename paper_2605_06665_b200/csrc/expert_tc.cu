@@ -13,8 +13,8 @@
 // UNIPOOL_ERR_TIMEOUT in the status word, all roles leave, TMEM is released.
 //   grouped_gemm_tc_kernel<MODE>  one CTA per 128 x 256 tile (cta_group::1), all six GEMMs
 //   wgrad_pair_kernel             the weight gradient on CTA pairs (cta_group::2, M = 256)
-//   row_pair_kernel<MODE>         gate/up, down and second dgrad on CTA pairs (M = 256, and M = 128
-//                                 for a group's odd last tile)
+//   row_pair_kernel<MODE>         the four row-tile GEMMs on CTA pairs (M = 256, and M = 128 for a
+//                                 group's odd last tile)
 #include <cuda.h>
 
 #include "common.cuh"
@@ -950,10 +950,20 @@ int map_chunk(const unipool_ctx* ctx, CUtensorMap* out, const void* base, uint64
 // Six operand stages and four epilogue warps: a variant with eight epilogue warps (two per TMEM lane
 // quarter, taking alternate chunks) had to give one stage to their staging tiles and was 8 - 12 %
 // slower - the main loop lives on the bytes it keeps in flight.
-constexpr int kRowPairStages = 6;
-constexpr int kRowPairEpiWarps = 4;
-constexpr int kRowPairThreads = 64 + 32 * kRowPairEpiWarps;
-static_assert(kRowPairStages * kPairStageBytes + kRowPairEpiWarps * 8192 == kBarOffset, "shared-memory budget");
+// The SwiGLU-derivative GEMM keeps its organisation of the single-CTA kernel (eight epilogue warps, one
+// operand mover per TMEM lane quarter, G and U turned into dG and dU in place in a ring of chunk
+// buffers): four operand stages, and a ring of six chunk pairs per quarter in the room the other two took.
+template <int MODE> struct PairTraits {
+  static constexpr bool kIo = MODE == kDgrad1;
+  static constexpr int kStages = kIo ? 4 : 6;
+  static constexpr int kEpiWarps = kIo ? 8 : 4;
+  static constexpr int kThreads = 64 + 32 * kEpiWarps + (kIo ? 128 : 0);
+  static constexpr uint32_t kStagingOffset = kStages * kPairStageBytes;
+  static constexpr uint32_t kStagingPerQuarter = kIo ? 24576 : 8192;
+  static_assert(kStagingOffset + 4 * kStagingPerQuarter == kBarOffset, "shared-memory budget");
+};
+constexpr int kPairRing = 6, kPairAhead = 3;           // dgrad1: ring slots per quarter, prefetch distance
+static_assert(kPairRing * 2 * kBf16ChunkBytes == PairTraits<kDgrad1>::kStagingPerQuarter, "ring size");
 
 // half: the pair-tile is ONE row tile (the odd last tile of a group): each CTA takes 64 of its rows and the
 // MMA is the M = 128 form of cta_group::2.
@@ -979,6 +989,44 @@ __device__ __forceinline__ PairTile pair_tile(const GemmParams& p, const uint16_
   return t;
 }
 
+// dgrad1 on pairs: the chunks (32 rows x 32 columns of dA) that the epilogue warps of TMEM lane quarter
+// `quarter` of CTA `rank` own in pair-tile t: first row, first column and how many (chunk i sits at TMEM
+// column 32 i under both accumulator layouts described below).
+__device__ __forceinline__ void pair_chunks(const GemmParams& p, const PairTile& t, int rank, int quarter, int& row0,
+                                            int& col0, int& nch) {
+  if (!t.half) {
+    row0 = (t.mt + rank) * BM + quarter * 32;
+    col0 = t.nt * BN;
+    nch = min(BN / kChunk, (p.f - col0) / kChunk);
+  } else {
+    row0 = t.mt * BM + rank * (BM / 2) + (quarter & 1) * 32;
+    col0 = t.nt * BN + (BN / 2) * (quarter >> 1);
+    nch = max(0, min(BN / 2 / kChunk, (p.f - col0) / kChunk));
+  }
+}
+
+// The (G, U) chunks of one lane quarter over all pair-tiles of this CTA pair, in the order the epilogue
+// consumes them (see ChunkCursor).
+struct PairChunkCursor {
+  int tile, ch, nch, col0, row0;
+  __device__ void seek(const GemmParams& p, const uint16_t* pp, int total, int n_nt, int total_q, int rank, int quarter) {
+    while (tile < total) {
+      pair_chunks(p, pair_tile(p, pp, tile, n_nt, total_q, false), rank, quarter, row0, col0, nch);
+      ch = 0;
+      if (nch > 0) return;
+      tile += gridDim.x >> 1;
+    }
+  }
+  __device__ void start(const GemmParams& p, const uint16_t* pp, int total, int n_nt, int total_q, int rank, int quarter) {
+    tile = blockIdx.x >> 1; ch = 0; nch = 0; col0 = 0; row0 = 0;
+    seek(p, pp, total, n_nt, total_q, rank, quarter);
+  }
+  __device__ void next(const GemmParams& p, const uint16_t* pp, int total, int n_nt, int total_q, int rank, int quarter) {
+    if (++ch == nch) { tile += gridDim.x >> 1; seek(p, pp, total, n_nt, total_q, rank, quarter); }
+  }
+  __device__ int col() const { return col0 + ch * kChunk; }
+};
+
 // Accumulator layouts (read back with tcgen05.ld, lanes [32 w, 32 w + 32) for warp w of a CTA):
 //   M = 256: the CTA's 128 rows are lanes 0..127, the tile's 256 columns TMEM columns 0..255;
 //   M = 128: the CTA's 64 rows are lanes 0..63 for columns 0..127 AND lanes 64..127 for columns
@@ -987,11 +1035,14 @@ __device__ __forceinline__ PairTile pair_tile(const GemmParams& p, const uint16_
 // half is [64 gate features | the same 64 up features], so that G and U of one element meet in one
 // thread under both layouts.
 template <int MODE>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kRowPairThreads, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(PairTraits<MODE>::kThreads, 1)
 row_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmA64,
                 const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmC0,
                 const __grid_constant__ CUtensorMap tmC1, const GemmParams p) {
-  static_assert(MODE == kFwd1 || MODE == kFwd2 || MODE == kDgrad2, "row tiles without epilogue operands");
+  static_assert(Traits<MODE>::kRowTiles, "row tiles");
+  using PT = PairTraits<MODE>;
+  constexpr int kRowPairStages = PT::kStages;
+  constexpr int kRowPairEpiWarps = PT::kEpiWarps;
   constexpr bool kBMn = Traits<MODE>::kBMn;
   constexpr bool kDescending = MODE == kFwd2 || MODE == kDgrad2;      // see tile_coord
   extern __shared__ uint8_t smem_raw[];
@@ -1000,8 +1051,11 @@ row_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   uint64_t* empty_bar = full_bar + kRowPairStages;
   uint64_t* tmem_full = empty_bar + kRowPairStages;
   uint64_t* tmem_empty = tmem_full + 2;
-  uint32_t* tmem_ptr = reinterpret_cast<uint32_t*>(tmem_empty + 2);
+  uint64_t* epi_bar = tmem_empty + 2;                        // dgrad1: [4][kPairRing] a chunk's G and U have landed
+  uint64_t* staged_bar = epi_bar + (PT::kIo ? 4 * kPairRing : 0);   // dgrad1: [4][kPairRing] dG and dU are staged
+  uint32_t* tmem_ptr = reinterpret_cast<uint32_t*>(staged_bar + (PT::kIo ? 4 * kPairRing : 0));
   volatile int* abort = reinterpret_cast<volatile int*>(tmem_ptr + 1);
+  static_assert((2 * PT::kStages + 4 + (PT::kIo ? 8 * kPairRing : 0)) * 8 + 8 <= 512, "barrier block");
   uint16_t* pp = reinterpret_cast<uint16_t*>(smem + kBarOffset + 512);       // [n_experts + 1]
 
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
@@ -1011,13 +1065,15 @@ row_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   if (threadIdx.x == 0) {
     for (int s = 0; s < kRowPairStages; ++s) { tc::mbar_init(&full_bar[s], 1); tc::mbar_init(&empty_bar[s], 1); }
     for (int a = 0; a < 2; ++a) { tc::mbar_init(&tmem_full[a], 1); tc::mbar_init(&tmem_empty[a], 2 * kRowPairEpiWarps); }
+    if constexpr (PT::kIo)
+      for (int i = 0; i < 4 * kPairRing; ++i) { tc::mbar_init(&epi_bar[i], 1); tc::mbar_init(&staged_bar[i], 1); }
     *abort = 0;
     tc::fence_barrier_init();
     tc::tma_prefetch_desc(&tmA);
     tc::tma_prefetch_desc(&tmA64);
     tc::tma_prefetch_desc(&tmB);
     tc::tma_prefetch_desc(&tmC0);
-    if constexpr (MODE == kFwd1) tc::tma_prefetch_desc(&tmC1);
+    if constexpr (MODE == kFwd1 || MODE == kDgrad1) tc::tma_prefetch_desc(&tmC1);
   }
   if (warp == 1) {
     tc::tmem_alloc_pair(tmem_ptr, 512);
@@ -1063,7 +1119,7 @@ row_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             tc::tma_load_3d_pair(sB, &tmB, &full_bar[stage], kb * BK, t.nt * (BN / 2) + rank * 64, 2 * pe);
           } else if constexpr (MODE == kFwd2) {    // 128 rows of W_down
             tc::tma_load_2d_pair(sB, &tmB, &full_bar[stage], kb * BK, pe * p.Ndim + t.nt * BN + rank * (BN / 2));
-          } else {                                 // two 64-column blocks of W_gu
+          } else {                                 // two 64-column blocks of the MN-major weights (W_down, W_gu)
             tc::tma_load_3d_pair(sB, &tmB, &full_bar[stage], 0, pe * p.Kdim + kb * BK, t.nt * 4 + rank * 2);
           }
           if (++stage == kRowPairStages) { stage = 0; phase ^= 1u; }
@@ -1108,13 +1164,60 @@ row_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         if (ok) tc::umma_commit_pair(&tmem_full[acc], 3);       // accumulator complete, both CTAs
       }
     }
+  } else if (PT::kIo && warp >= 2 + kRowPairEpiWarps) {
+    // ------------------------------------------------------------ dgrad1: operand mover of one lane quarter
+    // (one lane; see the single-CTA kernel: G and U are fetched kPairAhead chunks ahead into the quarter's
+    // ring and written back as dG, dU once the epilogue warps have rewritten them in place)
+    if constexpr (PT::kIo) {
+      if (lane == 0) {
+        const int ew = warp - (2 + kRowPairEpiWarps);
+        const int quarter = (ew + 2) & 3;
+        uint8_t* stg = smem + PT::kStagingOffset + ew * PT::kStagingPerQuarter;
+        uint64_t* full = epi_bar + kPairRing * ew;
+        uint64_t* staged = staged_bar + kPairRing * ew;
+        PairChunkCursor ld, st;
+        ld.start(p, pp, total, n_nt, total_q, rank, quarter);
+        st.start(p, pp, total, n_nt, total_q, rank, quarter);
+        int fetched = 0, stored = 0;
+        bool ok = true;
+        while (st.tile < total && ok) {
+          // Chunk n uses slot n % kPairRing.  When chunk `fetched` < stored + kPairAhead is fetched, the
+          // store that last read its slot (chunk fetched - kPairRing) is followed by at least
+          // kPairRing - kPairAhead committed stores: all but that many must have drained.
+          while (fetched < stored + kPairAhead && ld.tile < total) {
+            const int slot = fetched % kPairRing;
+            uint8_t* buf = stg + slot * 2 * kBf16ChunkBytes;
+            tc::bulk_wait_read<kPairRing - kPairAhead - 1>();
+            tc::mbar_expect_tx(&full[slot], 2 * kBf16ChunkBytes);
+            tc::tma_load_2d(buf, &tmC1, &full[slot], ld.col(), ld.row0);
+            tc::tma_load_2d(buf + kBf16ChunkBytes, &tmC1, &full[slot], p.f + ld.col(), ld.row0);
+            ++fetched;
+            ld.next(p, pp, total, n_nt, total_q, rank, quarter);
+          }
+          const int slot = stored % kPairRing;
+          uint8_t* buf = stg + slot * 2 * kBf16ChunkBytes;
+          if (!tc::mbar_wait(&staged[slot], (stored / kPairRing) & 1, abort)) { report_timeout(p, abort, 36); ok = false; break; }
+          tc::tma_store_2d(&tmC0, buf, st.col(), st.row0);
+          tc::tma_store_2d(&tmC0, buf + kBf16ChunkBytes, p.f + st.col(), st.row0);
+          tc::bulk_commit();
+          ++stored;
+          st.next(p, pp, total, n_nt, total_q, rank, quarter);
+        }
+        if (!ok)
+          for (int i = 0; i < 200; ++i) __nanosleep(1000);   // let loads already in flight land
+        tc::bulk_wait<0>();
+      }
+    }
   } else {
     // ------------------------------------------------------------ epilogue: this CTA's rows of the pair-tile
+    // (dgrad1: two warps per lane quarter, warps w and w + 4, share the quarter's ring and take alternate chunks)
     const int quarter = warp & 3;
-    uint8_t* stg = smem + kRowPairStages * kPairStageBytes + (warp - 2) * 8192;
+    const int ew = (warp - 2) & 3;
+    uint8_t* stg = smem + PT::kStagingOffset + ew * PT::kStagingPerQuarter;
     int gchunk = 0, local = 0;
     (void)gchunk;
-    for (int tile = pair; tile < total; tile += n_pairs) {
+    bool ok = true;
+    for (int tile = pair; tile < total && ok; tile += n_pairs) {
       const PairTile t = pair_tile(p, pp, tile, n_nt, total_q, kDescending);
       const int acc = local & 1;
       const uint32_t acc_phase = (local >> 1) & 1;
@@ -1125,7 +1228,46 @@ row_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       }
       tc::tc_fence_after_sync();
       const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * BN;
-      if (!t.half) {
+      if constexpr (MODE == kDgrad1) {
+        const int half = (warp - 2) >> 2;
+        uint64_t* my_bar = epi_bar + kPairRing * ew;
+        uint64_t* my_staged = staged_bar + kPairRing * ew;
+        int row0, col0, nch;
+        pair_chunks(p, t, rank, quarter, row0, col0, nch);
+#pragma unroll 1
+        for (int ch = 0; ch < nch; ++ch) {
+          if (((gchunk + ch) & 1) != half) continue;    // the other warp of this quarter takes it
+          const int slot = (gchunk + ch) % kPairRing;
+          const uint32_t slot_phase = ((gchunk + ch) / kPairRing) & 1;
+          uint8_t* buf = stg + slot * 2 * kBf16ChunkBytes;
+          uint32_t rr[32];
+          tc::tmem_ld_32x32(t_row + ch * kChunk, rr);
+          tc::tmem_ld_wait();
+          if (!tc::mbar_wait(&my_bar[slot], slot_phase, abort)) {
+            if (lane == 0) report_timeout(p, abort, 35);
+            ok = false;
+            break;
+          }
+          float g[32], u[32], dg[32], du[32];
+          unstage_row_bf16(buf, lane, g);
+          unstage_row_bf16(buf + kBf16ChunkBytes, lane, u);
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const float dA = __uint_as_float(rr[i]);
+            const float sig = sigmoid_fast(g[i]);
+            const float sl = g[i] * sig;
+            dg[i] = dA * u[i] * (sig + sl * (1.0f - sig));   // silu'(g) = sig (1 + g (1 - sig))
+            du[i] = dA * sl;
+          }
+          stage_row_bf16(buf, lane, dg);               // in place: each lane rewrites the row it read
+          stage_row_bf16(buf + kBf16ChunkBytes, lane, du);
+          tc::fence_proxy_async();
+          __syncwarp();
+          if (lane == 0) tc::mbar_arrive(&my_staged[slot]);   // the operand mover stores the chunk
+        }
+        gchunk += nch;
+        if (!ok) break;
+      } else if (!t.half) {
         const int row0 = (t.mt + rank) * BM + quarter * 32;
         if constexpr (MODE == kFwd1) {
 #pragma unroll 1
@@ -1140,7 +1282,7 @@ row_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         const int row0 = t.mt * BM + rank * (BM / 2) + (quarter & 1) * 32;
         if constexpr (MODE == kFwd1)
           epilogue_swiglu(&tmC0, &tmC1, p, t_row, t_row + 64, t.nt * (BN / 2) + 64 * h, 2, row0, stg, lane);
-        else
+        else if constexpr (MODE != kDgrad1)
           epilogue_rows<MODE>(&tmC0, p, t_row, t.nt * BN + 128 * h, BN / 2, row0, stg, lane, gchunk);
       }
       tc::tc_fence_before_sync();
@@ -1150,6 +1292,8 @@ row_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         else tc::mbar_arrive_leader(&tmem_empty[acc]);
       }
     }
+    if (!ok && lane == 0)
+      for (int i = 0; i < 200; ++i) __nanosleep(1000);       // let loads already in flight land before the CTA retires
     if (lane < 3) tc::bulk_wait<0>();
     __syncwarp();
   }
@@ -1197,7 +1341,7 @@ int launch_rows(unipool_ctx* ctx, int phase, bool pairs, const CUtensorMap& tmA,
   if (pairs) {
     auto kern = row_pair_kernel<MODE>;
     UP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPairSmemTotal));
-    kern<<<ctx->sm_count / 2 * 2, kRowPairThreads, kPairSmemTotal, s>>>(tmA, tmA64, tmBp, tmC0, tmC1, p);
+    kern<<<ctx->sm_count / 2 * 2, PairTraits<MODE>::kThreads, kPairSmemTotal, s>>>(tmA, tmA64, tmBp, tmC0, tmC1, p);
   } else {
     auto kern = grouped_gemm_tc_kernel<MODE>;
     UP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemTotal));
@@ -1317,16 +1461,21 @@ int expert_bwd_tc(unipool_ctx* ctx, const ExpertBwdArgs& a, cudaStream_t s) {
   p.expert_base = a.expert_base;
   p.f = f;
   p.status = ctx->ws.status;
-  CUtensorMap tmA, tmB, tmB64, tmBp, tmC0, tmC1;
+  p.group_offsets = a.offsets;
+  const bool plan = rows_on_pairs(ctx, a.n_experts);
+  CUtensorMap tmA, tmA64, tmB, tmB64, tmBp, tmC0, tmC1;
   int rc;
   // dA = dYp W_down, fused with the SwiGLU derivative -> dGU
   if ((rc = map_2d(ctx, &tmA, a.dYp, d, cap, 64, BM)) != UNIPOOL_OK) return rc;
+  if ((rc = map_2d(ctx, &tmA64, a.dYp, d, cap, 64, 64)) != UNIPOOL_OK) return rc;
   if ((rc = map_mn(ctx, &tmB, a.W_down, f, (uint64_t)M * d, BN / 64)) != UNIPOOL_OK) return rc;
+  if ((rc = map_mn(ctx, &tmBp, a.W_down, f, (uint64_t)M * d, BN / 128)) != UNIPOOL_OK) return rc;
   if ((rc = map_2d(ctx, &tmB64, a.W_down, f, (uint64_t)M * d, 64, 64)) != UNIPOOL_OK) return rc;
   if ((rc = map_chunk(ctx, &tmC0, a.dGU, 2 * f, cap, kMapBf16Chunk)) != UNIPOOL_OK) return rc;
   if ((rc = map_chunk(ctx, &tmC1, a.GU, 2 * f, cap, kMapBf16Chunk)) != UNIPOOL_OK) return rc;
   p.Ndim = f; p.Kdim = d;
-  if ((rc = launch<kDgrad1>(ctx, UNIPOOL_PH_DGRAD_DOWN, tmA, tmB, tmB64, tmC0, tmC1, p, s)) != UNIPOOL_OK) return rc;
+  rc = launch_rows<kDgrad1>(ctx, UNIPOOL_PH_DGRAD_DOWN, plan, tmA, tmA64, tmB, tmB64, tmBp, tmC0, tmC1, p, s);
+  if (rc != UNIPOOL_OK) return rc;
   // dXp = dGU [W_gate; W_up]
   if ((rc = map_2d(ctx, &tmA, a.dGU, 2 * f, cap, 64, BM)) != UNIPOOL_OK) return rc;
   if ((rc = map_mn(ctx, &tmB, a.W_gu, d, (uint64_t)M * 2 * f, BN / 64)) != UNIPOOL_OK) return rc;
@@ -1334,11 +1483,8 @@ int expert_bwd_tc(unipool_ctx* ctx, const ExpertBwdArgs& a, cudaStream_t s) {
   if ((rc = map_2d(ctx, &tmB64, a.W_gu, d, (uint64_t)M * 2 * f, 64, 64)) != UNIPOOL_OK) return rc;
   if ((rc = map_chunk(ctx, &tmC0, a.dXp, d, cap, kMapBf16Chunk)) != UNIPOOL_OK) return rc;
   p.Ndim = d; p.Kdim = 2 * f; p.overwrite = 1;
-  p.group_offsets = a.offsets;
-  CUtensorMap tmA64;
   if ((rc = map_2d(ctx, &tmA64, a.dGU, 2 * f, cap, 64, 64)) != UNIPOOL_OK) return rc;
-  rc = launch_rows<kDgrad2>(ctx, UNIPOOL_PH_DGRAD_GU, rows_on_pairs(ctx, a.n_experts), tmA, tmA64, tmB, tmB64, tmBp, tmC0,
-                            tmC0, p, s);
+  rc = launch_rows<kDgrad2>(ctx, UNIPOOL_PH_DGRAD_GU, plan, tmA, tmA64, tmB, tmB64, tmBp, tmC0, tmC0, p, s);
   if (rc != UNIPOOL_OK) return rc;
   if (a.wgrad) {
     PoolWgradArgs w{1, 0, a.offsets, a.Xp, a.A, a.dYp, a.dGU, a.expert_base, a.n_experts, a.dW_gu, a.dW_down,

@@ -169,7 +169,7 @@ def test_small_fp32_shapes(kw, T):
     (dict(dtype="bf16", d=128, f=128, M=10, k=3), 333),     # logit rows that are not 16-byte aligned
     (dict(dtype="bf16", d=64, f=64, M=512, k=8), 257),      # the largest pool and top-k, the smallest widths
     (dict(dtype="bf16", d=128, f=192, M=16, k=2), 1),       # a single token
-    # groups of several row tiles: the forward GEMMs and the second dgrad run on CTA pairs
+    # groups of several row tiles: the four row-tile GEMMs run on CTA pairs
     (dict(dtype="bf16", d=256, f=320, M=4, k=2, zipf_beta=1.0), 2100),   # skewed: odd and even tile counts, f % 128 = 64
     (dict(dtype="bf16", d=192, f=256, M=2, k=1), 2500),                  # d % 256 = 192: a clipped last column tile
     (dict(dtype="bf16", d=256, f=256, M=6, k=2, private=2, L=3), 1100),  # private experts through pool views
