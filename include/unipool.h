@@ -109,7 +109,14 @@ const char* unipool_last_error(void);
 
 /* Reads the context's device status word (the one call that synchronises
  * `stream`).  Returns UNIPOOL_OK, UNIPOOL_ERR_TIMEOUT or
- * UNIPOOL_ERR_DEVICE_CHECK and clears the word. */
+ * UNIPOOL_ERR_DEVICE_CHECK and clears the word.
+ * Debug mode: when the environment holds UNIPOOL_DEBUG=1 at the first call
+ * into the library, every region of the workspace is followed by a 256-byte
+ * guard band (unipool_workspace_bytes() grows by 256 per region) filled by
+ * unipool_create(); this call first compares the bands with their fill (one
+ * small launch on `stream`) and reports an altered one as
+ * UNIPOOL_ERR_DEVICE_CHECK, unipool_last_error() naming the region.  The
+ * paper has no counterpart: a development aid. */
 int unipool_check_status(unipool_ctx* ctx, unipool_stream stream);
 
 /* NormRouter scoring and top-k of one layer (Eq. 7; Sec. 4.3 "Top-k selection").

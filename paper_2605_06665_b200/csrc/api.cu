@@ -23,6 +23,15 @@ static bool use_tensor_cores(const unipool_ctx* ctx) { return ctx->cfg.dtype == 
 
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// UNIPOOL_DEBUG=1 in the environment (read once per process): guard bands behind the workspace regions
+static bool debug_enabled() {
+  static const bool on = [] {
+    const char* v = getenv("UNIPOOL_DEBUG");
+    return v != nullptr && v[0] == '1' && v[1] == '\0';
+  }();
+  return on;
+}
+
 static int64_t row_capacity_of(const unipool_config& c) {
   int64_t rows = (int64_t)c.max_tokens * c.top_k + (int64_t)c.pool_size * (UNIPOOL_ROW_ALIGN - 1);
   return (rows + UNIPOOL_ROW_ALIGN - 1) / UNIPOOL_ROW_ALIGN * UNIPOOL_ROW_ALIGN;
@@ -32,9 +41,14 @@ Workspace carve_workspace(const unipool_config& cfg, void* base) {
   Workspace w{};
   size_t off = 0;
   char* p = static_cast<char*>(base);
+  const bool guarded = debug_enabled();
   auto take = [&](size_t bytes) {
     char* q = p ? p + off : nullptr;
     off += align_up(bytes, 256);
+    if (guarded && w.n_guards < 16) {
+      w.guards[w.n_guards++] = p ? p + off : nullptr;
+      off += kGuardBytes;
+    }
     return q;
   };
   const size_t eb = cfg.dtype == UNIPOOL_BF16 ? 2 : 4;
@@ -144,6 +158,8 @@ int unipool_create(unipool_ctx** out, const unipool_config* cfg, void* workspace
   // the self-cleaning accumulators and the status word start at zero
   size_t head = reinterpret_cast<char*>(w.block_hist) - reinterpret_cast<char*>(workspace);
   if (e == cudaSuccess) e = cudaMemsetAsync(workspace, 0, head, static_cast<cudaStream_t>(stream));
+  for (int i = 0; i < w.n_guards && e == cudaSuccess; ++i)
+    e = cudaMemsetAsync(w.guards[i], (int)(kGuardWord & 0xff), kGuardBytes, static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) {
     set_error("context set-up failed: %s", cudaGetErrorString(e));
     delete ctx;
@@ -195,6 +211,10 @@ int unipool_check_status(unipool_ctx* ctx, unipool_stream stream) {
   CHECK_CTX(ctx);
   int32_t host[4] = {0, 0, 0, 0};
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (ctx->ws.n_guards > 0) {
+    int rc = guard_check_launch(ctx, s);
+    if (rc != UNIPOOL_OK) return rc;
+  }
   UP_CUDA(cudaMemcpyAsync(host, ctx->ws.status, sizeof(host), cudaMemcpyDeviceToHost, s));
   UP_CUDA(cudaStreamSynchronize(s));
   if (host[0] == 0) return UNIPOOL_OK;
@@ -204,7 +224,10 @@ int unipool_check_status(unipool_ctx* ctx, unipool_stream stream) {
     set_error("a bounded device-side wait ran out (site %d, detail %d)", host[1], host[2]);
     return UNIPOOL_ERR_TIMEOUT;
   }
-  set_error("device-side consistency check failed (site %d, detail %d)", host[1], host[2]);
+  if (host[1] >= kGuardSite && host[1] < kGuardSite + 16)
+    set_error("the guard band behind workspace region %d was overwritten (byte %d of it)", host[1] - kGuardSite, host[2]);
+  else
+    set_error("device-side consistency check failed (site %d, detail %d)", host[1], host[2]);
   return UNIPOOL_ERR_DEVICE_CHECK;
 }
 

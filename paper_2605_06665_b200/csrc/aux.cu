@@ -173,6 +173,24 @@ __global__ void wait_selftest_kernel(long long limit_cycles, int32_t* status) {
   }
 }
 
+// Debug mode: one block per guard band, a thread per word; the first band found altered is reported in
+// the status word (site kGuardSite + band, detail = byte offset inside the band).
+struct GuardList { const unsigned* band[16]; };
+__global__ void guard_check_kernel(GuardList gl, int32_t* status) {
+  if (gl.band[blockIdx.x][threadIdx.x] != kGuardWord && atomicCAS(status, 0, kStatusCheck) == 0) {
+    status[1] = kGuardSite + (int)blockIdx.x;
+    status[2] = (int)threadIdx.x * 4;
+  }
+}
+
+int guard_check_launch(unipool_ctx* ctx, cudaStream_t s) {
+  GuardList gl{};
+  for (int i = 0; i < ctx->ws.n_guards; ++i) gl.band[i] = reinterpret_cast<const unsigned*>(ctx->ws.guards[i]);
+  guard_check_kernel<<<ctx->ws.n_guards, kGuardBytes / 4, 0, s>>>(gl, ctx->ws.status);
+  UP_LAUNCH_CHECK();
+  return UNIPOOL_OK;
+}
+
 int wait_selftest_launch(unipool_ctx* ctx, long long limit_cycles, cudaStream_t s) {
   wait_selftest_kernel<<<1, 32, 0, s>>>(limit_cycles, ctx->ws.status);
   UP_LAUNCH_CHECK();

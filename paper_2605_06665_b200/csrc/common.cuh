@@ -60,7 +60,12 @@ struct Workspace {
   float*   part_dsigma;   // [ceil(max_tokens/64)] per-block dsigma terms
   void*    dXp;           // [row_capacity, d] expert_bwd scratch (ctx dtype)
   size_t   bytes;         // total
+  char*    guards[16];    // debug mode: the 256-byte guard band behind each region
+  int      n_guards;      // 0 unless UNIPOOL_DEBUG=1
 };
+constexpr int kGuardBytes = 256;
+constexpr unsigned kGuardWord = 0xA5A5A5A5u;
+constexpr int kGuardSite = 200;               // status site of guard band i: kGuardSite + i
 
 constexpr int kDispatchChunkTokens = 256;     // most tokens per block of the permute kernels (eight warps of 32)
 constexpr int kDispatchMinChunkTokens = 64;   // fewest
@@ -156,6 +161,7 @@ int aux_launch(unipool_ctx*, const int32_t* counts, const float* S, int L, int n
 int unique_experts_launch(unipool_ctx*, const int32_t* idx, const int32_t* expert_base, int L, int T,
                           int32_t* unique, unsigned long long* total, cudaStream_t);
 int wait_selftest_launch(unipool_ctx*, long long limit_cycles, cudaStream_t);
+int guard_check_launch(unipool_ctx*, cudaStream_t);
 int calibrate_launch(unipool_ctx*, int n_experts, int top_k, int n_samples, uint64_t seed,
                      float* c_out, cudaStream_t);
 

@@ -59,3 +59,22 @@ def test_missing_workspace_is_refused(lib):
 def test_null_context_is_refused(lib):
     assert lib.unipool_check_status(None, None) == -1
     assert lib.unipool_destroy(None) == 0
+
+
+def test_debug_mode_adds_a_guard_band_per_workspace_region(lib):
+    """UNIPOOL_DEBUG=1 (read once per process, hence the child): 256 bytes behind each of the 13
+    regions of a bf16 workspace, 12 of an fp32 one (no split router weights there)."""
+    import subprocess
+    import sys
+    code = (
+        "from paper_2605_06665_b200 import binding as B\n"
+        "for dt in (B.BF16, B.FP32):\n"
+        "    print(B.workspace_bytes(B.make_config(256, 512, 16, 2, 4, 512, dt, 1e-6, 2.0)))\n"
+    )
+    sizes = {}
+    for flag in ("0", "1"):
+        env = dict(os.environ, UNIPOOL_DEBUG=flag)
+        out = subprocess.run([sys.executable, "-c", code], cwd=ROOT, env=env, capture_output=True, text=True, check=True)
+        sizes[flag] = [int(v) for v in out.stdout.split()]
+    assert sizes["1"][0] - sizes["0"][0] == 13 * 256
+    assert sizes["1"][1] - sizes["0"][1] == 12 * 256

@@ -5,6 +5,8 @@ Tolerances (max|gpu - ref| / max|ref|): 1e-5 in fp32 mode, 1e-2 for bf16 storage
 with fp32 accumulation; balance loss relative 1e-5; routing indices, counts and
 the permutation maps bit-exact (indices: where the logit margin exceeds 1e-4).
 """
+import os
+
 import numpy as np
 import pytest
 
@@ -649,3 +651,44 @@ def test_an_expired_device_wait_is_reported_and_the_context_stays_usable():
         st.ctx.selftest_wait(-1)                     # refused on the host
     st.close()
 
+
+
+_GUARD_CHILD = r"""
+import numpy as np, torch
+from paper_2605_06665_b200 import binding as B, synth
+from paper_2605_06665_b200.stack import UniPoolStack
+cfg = dict(synth.CONFIGS["tiny_fp32"]); cfg.update(dtype="bf16", d=128, f=128, M=8, k=2, L=2, T=300)
+inp = synth.make_inputs(cfg, seed=5)
+st = UniPoolStack(cfg["L"], cfg["d"], cfg["f"], cfg["M"], cfg["k"], cfg["T"], "bf16", 0, c=2.0, device="cuda:0")
+st.load(inp["pool"], inp["routers"])
+x0 = torch.from_numpy(inp["x0"]).to("cuda:0", torch.bfloat16)
+y = st.forward(x0)
+st.aux_loss()
+st.backward(torch.ones_like(y))
+st.ctx.check_status()                       # a whole step leaves every band as it was filled
+print("intact")
+ws = st.ctx.workspace
+assert int(ws[256]) == 0xA5                 # the first band follows the 256-byte status region
+ws[300] = 0                                 # what a kernel writing past its region would do
+try:
+    st.ctx.check_status()
+    print("missed")
+except B.UniPoolError as e:
+    print("caught", e.code, str(e))
+st.ctx.check_status()                       # reported once, the word is cleared; the band stays altered
+"""
+
+
+@pytest.mark.gpu
+def test_debug_guard_bands_survive_a_step_and_report_an_overwrite():
+    """Debug aid (no paper counterpart): with UNIPOOL_DEBUG=1 the workspace regions are fenced by
+    guard bands that unipool_check_status compares with their fill."""
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, UNIPOOL_DEBUG="1")
+    out = subprocess.run([sys.executable, "-c", _GUARD_CHILD], cwd=root, env=env, capture_output=True, text=True)
+    assert out.returncode != 0 or "intact" in out.stdout, out.stderr[-2000:]
+    lines = out.stdout.strip().splitlines()
+    assert lines[0] == "intact", out.stdout + out.stderr[-2000:]
+    assert lines[1].startswith("caught -6") and "guard band behind workspace region 0" in lines[1], out.stdout
