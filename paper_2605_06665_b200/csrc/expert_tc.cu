@@ -1318,7 +1318,7 @@ int launch(unipool_ctx* ctx, int phase, const CUtensorMap& tmA, const CUtensorMa
   return UNIPOOL_OK;
 }
 
-// The row-tile GEMMs (gate/up, down, second dgrad) of a call run either all on the single-CTA kernel or
+// The four row-tile GEMMs (gate/up, down, both dgrads) of a call run either all on the single-CTA kernel or
 // all on CTA pairs (the odd last tile of a group as a half pair-tile, M = 128).  Pairs move a third
 // fewer operand bytes into the SMs.  Measured (interleaved runs, one B200), pairs against single per
 // GEMM: -10 % at 32 row tiles per group, -3 .. -8 % at 4 - 7 tiles, none at 2.7 tiles (341 rows): a
