@@ -55,6 +55,8 @@ CONFIGS = {
     # layer's full token batch over an eighth of the pool (activations larger than the L2 cache)
     "978m_slice":     dict(L=1,  d=1536, f=4096, M=24,  k=2, T=4096,  dtype="bf16", private=0, zipf_beta=0.0),
     "978m_tokens":    dict(L=1,  d=1536, f=4096, M=24,  k=2, T=32768, dtype="bf16", private=0, zipf_beta=0.0),
+    # one private layer of eight experts at a quarter of its tokens: groups of ~16 row tiles (the CTA-pair kernels)
+    "978m_groups":    dict(L=1,  d=1536, f=4096, M=8,   k=2, T=8192,  dtype="bf16", private=0, zipf_beta=0.0),
     "fine_zipf":      dict(L=12, d=768,  f=512,  M=384, k=8, T=16384, dtype="bf16", private=0, zipf_beta=0.4),
 }
 
