@@ -301,14 +301,19 @@ def measure_workload(name, args, world, rank, dev, full):
     gemm_ms = {n: kernels[n]["ms_per_step"] for n in GEMM_PHASES if n in kernels}
     dominant = max(gemm_ms, key=gemm_ms.get)
     dom = kernels[dominant]
+    # the library runs the row-tile GEMMs on CTA pairs when a full batch gives the average expert of a
+    # layer's view four row tiles of 128 rows
+    kernel_name = GEMM_KERNEL[dominant]
+    if kernel_name == "grouped_gemm_tc_kernel" and T * k >= 4 * 128 * mw:
+        kernel_name = "row_pair_kernel"
     # per launch of the dominant kernel: algorithmic bytes / FLOPs over its average CUDA-event duration
     if dom["bound"] == "hbm":
-        roofline = dict(kernel=GEMM_KERNEL[dominant] + ":" + dominant, bound="hbm", achieved=dom["gbs"],
+        roofline = dict(kernel=kernel_name + ":" + dominant, bound="hbm", achieved=dom["gbs"],
                         peak=peaks["hbm_gbs"], unit="GB/s", frac=dom["gbs"] / peaks["hbm_gbs"],
                         peak_source=peaks["source"], traffic=None,
                         tensor_tflops=dom["tflops"], tensor_frac_of_sustained=dom["frac_of_measured_sustained"])
     else:
-        roofline = dict(kernel=GEMM_KERNEL[dominant] + ":" + dominant, bound="tensor", achieved=dom["tflops"],
+        roofline = dict(kernel=kernel_name + ":" + dominant, bound="tensor", achieved=dom["tflops"],
                         peak=peaks["bf16_tflops_sustained"], unit="TFLOP/s",
                         frac=dom["tflops"] / peaks["bf16_tflops_sustained"],
                         peak_source=peaks["source"] + " sustained", traffic=None, hbm_gbs=dom["gbs"])
