@@ -409,61 +409,79 @@ def run_ours(args):
         print(json.dumps(out))
 
 
-def cpu_baseline(cfg, budget_tokens=2048, repeats=1):
-    """Times the CPU oracle, as it stands, on one MoE layer (forward + backward) over a
-    token sample of the workload; fp32 arithmetic (the arrays it is fed are float32)."""
+def oracle_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        return int(max([p.get("num_threads", 1) for p in threadpool_info()] or [1]))
+    except Exception:
+        return len(os.sched_getaffinity(0))
+
+
+def oracle_layer_step(cfg, inputs, Ts):
+    """One MoE layer (forward, balance-loss term, backward with all gradients) of the CPU oracle, as it
+    stands, over the first Ts tokens of `inputs`; float32 arithmetic (the arrays it is fed are float32).
+    Returns the seconds it took."""
     import numpy as np
     from oracle import unipool_oracle as O
     from paper_2605_06665_b200 import synth
-    try:
-        from threadpoolctl import threadpool_info
-        threads = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
-    except Exception:
-        threads = len(os.sched_getaffinity(0))
-    Ts = min(budget_tokens, cfg["T"])
-    inputs = synth.make_inputs(cfg, seed=0, T=Ts, L=1)
     pool, router = inputs["pool"], dict(inputs["routers"][0], mode=cfg.get("router", "norm"))
     k = cfg["k"]
-    best = None
-    for _ in range(repeats):
-        t0 = time.perf_counter()
-        cache = O.layer_forward(inputs["x0"], router, pool, k, np.float32(2.0), np.float32(synth.EPS))
-        _, _, coef = O.pool_aux_loss(cache["counts"][None], cache["S"][None], Ts, k, synth.ALPHA)
-        grad = O.zeros_like_pool(pool)
-        O.layer_backward(cache, router, pool, k, np.float32(2.0), np.float32(synth.EPS), inputs["upstream"],
-                         coef.astype(np.float32), grad)
-        dt = time.perf_counter() - t0
-        best = dt if best is None else min(best, dt)
-    return dict(value=Ts / best, unit=UNIT, cores=int(threads), kind="oracle", seconds=best,
-                sample=f"one MoE layer fwd+bwd (route, Eq. 2, balance-loss term, all gradients) over {Ts} of the "
-                       f"{cfg['T']} tokens, full pool of {cfg['M']} experts, float32 numpy")
+    t0 = time.perf_counter()
+    cache = O.layer_forward(inputs["x0"][:Ts], router, pool, k, np.float32(2.0), np.float32(synth.EPS))
+    _, _, coef = O.pool_aux_loss(cache["counts"][None], cache["S"][None], Ts, k, synth.ALPHA)
+    grad = O.zeros_like_pool(pool)
+    O.layer_backward(cache, router, pool, k, np.float32(2.0), np.float32(synth.EPS), inputs["upstream"][:Ts],
+                     coef.astype(np.float32), grad)
+    return time.perf_counter() - t0
+
+
+def oracle_sample_text(cfg, Ts):
+    return (f"one MoE layer fwd+bwd (route, Eq. 2, balance-loss term, all gradients) over {Ts} of the "
+            f"{cfg['T']} tokens, full pool of {cfg['M']} experts, float32 numpy")
+
+
+def cpu_baseline(cfg, budget_tokens=2048):
+    """Times the CPU oracle on one MoE layer over a token sample of the workload."""
+    from paper_2605_06665_b200 import synth
+    Ts = min(budget_tokens, cfg["T"])
+    inputs = synth.make_inputs(cfg, seed=0, T=Ts, L=1)
+    sec = oracle_layer_step(cfg, inputs, Ts)
+    return dict(value=Ts / sec, unit=UNIT, cores=oracle_threads(), kind="oracle", seconds=sec,
+                sample=oracle_sample_text(cfg, Ts))
 
 
 def run_reference(args):
-    """The reference arm is the oracle (the paper ships no implementation)."""
+    """The reference arm is the oracle (the paper ships no implementation): W warm-up steps, then exactly K
+    timed steps, each one layer over the same token sample; the sample is halved until the projected run
+    fits the time budget."""
     from paper_2605_06665_b200 import synth
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     import __graft_entry__ as entry  # noqa: F401  (path set-up)
     cfg = dict(synth.CONFIGS[args.workload])
-    for _ in range(min(args.warmup, 1)):
-        cpu_baseline(cfg, budget_tokens=min(256, args.cpu_tokens))
-    times = []
-    res = None
-    for _ in range(min(args.steps, 3)):
-        res = cpu_baseline(cfg, budget_tokens=args.cpu_tokens)
-        times.append(res["seconds"])
-    sec = sum(times) / len(times)
-    Ts = min(args.cpu_tokens, cfg["T"])
+    Ts = min(args.ref_tokens, cfg["T"])
+    inputs = synth.make_inputs(cfg, seed=0, T=Ts, L=1)
+    n_total = args.steps + max(args.warmup, 1)
+    first = oracle_layer_step(cfg, inputs, Ts)                      # warm-up step 1, also the probe
+    while first * n_total > args.ref_budget_s and Ts > 256:
+        Ts //= 2
+        first = oracle_layer_step(cfg, inputs, Ts)
+    for _ in range(args.warmup - 1):
+        oracle_layer_step(cfg, inputs, Ts)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_layer_step(cfg, inputs, Ts)
+    sec = (time.perf_counter() - t0) / max(args.steps, 1)
     value = Ts / sec
     out = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT,
-        "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": len(times), "warmup": min(args.warmup, 1),
+        "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
         "config": {"workload": args.workload, "note": "CPU oracle; each step = one MoE layer fwd+bwd over a token sample"},
-        "cpu_baseline": {k: res[k] for k in ("value", "unit", "cores", "kind", "sample")},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
+                         "sample": oracle_sample_text(cfg, Ts)},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(out))
@@ -483,6 +501,9 @@ def main():
                     help="accumulate each layer's weight gradient into the pool gradient during that layer's "
                          "backward instead of contracting all layers' rows per expert in one pass at the end")
     ap.add_argument("--cpu-tokens", type=int, default=16384, help="token sample of the CPU-oracle baseline")
+    ap.add_argument("--ref-tokens", type=int, default=4096,
+                    help="--impl reference: tokens per step of the oracle (halved while the run would exceed the budget)")
+    ap.add_argument("--ref-budget-s", type=float, default=240.0, help="--impl reference: time budget of the whole run")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--grad-exchange", action="store_true",
                     help="also time the data-parallel step (routing statistics and gradients summed over the "
